@@ -1,0 +1,164 @@
+/*
+ * moe_apk.h -- C ABI of the B200 (sm_100a) routed-MoE expert library.
+ *
+ * One "operation" is the routed-expert computation of one token batch of one class
+ * (decode or prefill) for one MoE layer:
+ *
+ *     y[t,:] = sum_j w[t,j] * FFN_{ids[t,j]}(x[t,:]),
+ *     FFN_e(x) = (silu(x W_gate[e]) * (x W_up[e])) W_down[e]
+ *
+ * (the paper's Section 2.1 MoE module; the kernel that runs it is the adaptive
+ * persistent kernel of Section 4: two grouped GEMMs, the activation, the MoE pre- and
+ * post-processing and the tile scheduler in one launch, Section 6.1).
+ *
+ * Conventions
+ *   - Every pointer in moe_op_t and the workspace is a DEVICE pointer owned by the
+ *     caller; the library never frees it and keeps no reference after moe_destroy.
+ *     moe_config_t / moe_op_t themselves, and all `out` arguments, are HOST memory.
+ *   - `stream` is a cudaStream_t passed as void*.  Calls only enqueue work; none of
+ *     them synchronises the host except moe_status and moe_read_tile_log.
+ *   - Row-major everywhere.  bf16 = 2-byte bfloat16, e4m3 = 1-byte OCP E4M3FN.
+ *   - Return value: 0 on success, a negative MOE_E* code otherwise.  Errors that only
+ *     the device can see (an expert id out of range, a wait that ran out) are recorded
+ *     in a device status word and read back with moe_status after a stream sync; a
+ *     kernel that hits one stops claiming tiles and returns -- it never traps or hangs.
+ *   - There is no CPU fallback: without a CUDA device every compute entry point fails
+ *     with MOE_ECUDA.
+ */
+#ifndef MOE_APK_H_
+#define MOE_APK_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  MOE_OK = 0,
+  MOE_EINVAL = -1,   /* bad argument: NULL, shape, alignment, slot out of range          */
+  MOE_ENOSPC = -2,   /* workspace too small / op larger than max_tokens_per_op           */
+  MOE_ECUDA = -3,    /* a CUDA runtime or driver call failed (no device, launch error)   */
+  MOE_ETIMEOUT = -4, /* device: a wait (ready word, dependency, pipeline) ran out        */
+  MOE_EBADID = -5,   /* device: an expert id outside [0, n_experts)                      */
+  MOE_EBOUNDS = -6,  /* device: an index check failed inside a kernel                    */
+  MOE_ENOTPLANNED = -7 /* moe_run / moe_combine on a slot with no moe_plan               */
+};
+
+enum { MOE_DTYPE_BF16 = 0, MOE_DTYPE_FP8_E4M3 = 1 };
+enum { MOE_CLASS_DECODE = 0, MOE_CLASS_PREFILL = 1 };
+
+/* Height of a token-dimension tile (the M_t of the footprint formula, Section 5.2). */
+#define MOE_TILE_M 128
+
+typedef struct moe_ctx moe_ctx_t; /* opaque, host side */
+
+typedef struct {
+  int32_t n_experts;         /* E, 1..1024                                               */
+  int32_t top_k;             /* k, 1..32                                                 */
+  int32_t hidden;            /* H, multiple of 256                                       */
+  int32_t inter;             /* I, multiple of 128                                       */
+  int32_t dtype;             /* MOE_DTYPE_*                                              */
+  int32_t max_tokens_per_op; /* sizes the per-slot scratch; buffers are fixed up front,  */
+  int32_t max_ops;           /* as the paper's preallocated final buffers (Section 4.4)  */
+  int32_t wait_limit_us;     /* device-side wait budget before MOE_ETIMEOUT; 0 = 2 s     */
+  int32_t tile_log_entries;  /* capacity of the per-tile log; 0 = logging off            */
+  int32_t n_ctas;            /* persistent grid size; 0 = one CTA per SM                 */
+} moe_config_t;
+
+typedef struct {
+  int32_t cls;      /* MOE_CLASS_DECODE (priority) or MOE_CLASS_PREFILL                   */
+  int32_t n_tokens; /* T >= 0                                                             */
+  const void* x;          /* [T, H] bf16 | e4m3                                           */
+  const float* x_scale;   /* [T, H/128] fp32 (e4m3 only, else NULL)                       */
+  const int32_t* topk_ids;/* [T, k] expert ids                                            */
+  const float* topk_w;    /* [T, k] router weights                                        */
+  const void* w_gate_up;  /* [E, 2I, H]: rows 0..I-1 gate, I..2I-1 up; K (=H) contiguous  */
+  const void* w_down;     /* [E, H, I]; K (=I) contiguous                                 */
+  const float* s_gate_up; /* [E, 2I/128, H/128] fp32 block scales (e4m3 only, else NULL)  */
+  const float* s_down;    /* [E, H/128, I/128]                                            */
+  void* y;                /* [T, H] bf16 output                                           */
+  int32_t* counts;        /* [E]    out: rows per expert                                  */
+  int32_t* offsets;       /* [E+1]  out: exclusive prefix sum, offsets[E] = T*k           */
+  int32_t* sorted_to_flat;/* [T*k]  out: packed row p -> flat routed index i = t*k + j    */
+  int32_t* flat_to_sorted;/* [T*k]  out: inverse permutation                              */
+  const uint32_t* ready;  /* optional: the op may be scheduled once *ready != 0           */
+  uint32_t* done;         /* optional: set to 1 when the op's last tile has committed     */
+  int32_t after_op;       /* -1, or a slot (of the same moe_run) that must finish first   */
+} moe_op_t;
+
+/* One record per executed tile (only when tile_log_entries > 0). Times are GPU
+ * globaltimer nanoseconds; the preemption-interval analysis of Section 6.5 is made
+ * from these. */
+typedef struct {
+  uint64_t t_claim;  /* the tile was taken from its queue                                 */
+  uint64_t t_commit; /* its outputs are written and published                             */
+  int32_t slot;      /* op slot                                                           */
+  int32_t tile;      /* index in the op's tile list                                       */
+  int16_t cls, kind; /* class; 0 = gate/up GEMM + SwiGLU, 1 = down GEMM, 2 = combine      */
+  int16_t cta, sm;   /* CTA index and SM id that ran it                                   */
+} moe_tile_rec_t;
+
+/* Bytes of device workspace moe_create needs for this configuration. */
+int moe_workspace_bytes(const moe_config_t* cfg, size_t* out);
+
+/* Builds a context on the current device.  dev_workspace: device memory, 1024-byte
+ * aligned, at least moe_workspace_bytes(); the library zeroes what it needs (on the
+ * legacy default stream, synchronously). */
+int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_ctx_t** out);
+void moe_destroy(moe_ctx_t* ctx);
+
+/* Plan (pre-processing): top-k ids -> counts, exclusive offsets by a device prefix
+ * sum, the stable permutation (rows of an expert keep ascending flat index -- the
+ * packed per-expert layout of Section 2.3), and the op's tile table, whose length is
+ * the footprint x_moe = sum_{e: m_e>0} ceil(m_e / M_t) of Section 5.2.  Binds `op` to
+ * `slot`; the struct is copied, the buffers it names must stay valid until the work
+ * enqueued on them has finished. */
+int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
+
+/* The persistent expert kernel over the planned ops in `slots` (one launch): every CTA
+ * repeatedly claims the next tile from the decode queue or the prefill queue of
+ * Section 4.2 -- CTAs with index below the decode budget prefer decode tiles, the
+ * others prefill tiles, each falling back to the other class when its own has nothing
+ * ready (Section 5.4) -- and runs it: gate/up grouped GEMM with fused SwiGLU, then the
+ * down grouped GEMM, on rows gathered through the permutation.  A phase switch happens
+ * only between tiles (Section 4.2), so results do not depend on the schedule.
+ * Ops of one class are served in the order given.  With fuse_combine != 0 the
+ * router-weighted combine runs as tiles of the same launch and y is final when the
+ * kernel ends; otherwise call moe_combine. */
+int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, void* stream);
+
+/* Post-processing: y[t,:] = sum_j w[t,j] * D[flat_to_sorted[t*k+j],:], slots added in
+ * order j = 0..k-1 in fp32 (Section 2.1, "combines their outputs"). */
+int moe_combine(moe_ctx_t* ctx, int slot, void* stream);
+
+/* Decode SM budget q of Section 5.4: a stream-ordered 4-byte write to the device word
+ * the running kernel reads at every tile boundary.  0 <= decode_sms. */
+int moe_set_budget(moe_ctx_t* ctx, int decode_sms, void* stream);
+
+/* Device status (synchronous copy; call after synchronising the stream).  code is 0 or
+ * a MOE_E* value; detail[0..3] describe where (meaning depends on code).  Clears it. */
+int moe_status(moe_ctx_t* ctx, int32_t* code, int32_t detail[4]);
+
+/* Footprint of a planned slot: x_moe (tiles of height MOE_TILE_M) and the number of
+ * queue entries.  Synchronous copy; call after synchronising the stream. */
+int moe_footprint(moe_ctx_t* ctx, int slot, int32_t* x_moe, int32_t* n_tiles);
+
+/* Copies the slot's tile table (x_moe entries of {expert, first packed row, rows, 0})
+ * to host memory.  Synchronous. */
+int moe_read_tile_table(moe_ctx_t* ctx, int slot, int32_t* host_out, int max_tiles);
+
+/* Copies up to max_records tile records of the last moe_run to host memory and
+ * returns how many were written in *n.  Synchronous. */
+int moe_read_tile_log(moe_ctx_t* ctx, moe_tile_rec_t* host_out, int max_records, int* n);
+
+/* Multiprocessor count of the context's device (the default persistent grid). */
+int moe_sm_count(moe_ctx_t* ctx);
+
+const char* moe_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MOE_APK_H_ */

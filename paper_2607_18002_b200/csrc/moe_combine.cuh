@@ -1,0 +1,44 @@
+// Router-weighted combine (post-processing): y[t,:] = sum_j w[t,j] * D[flat_to_sorted[t*k+j],:]
+// with the k slots added in order in fp32 (Section 2.1 of the paper: the module "combines
+// their outputs").  One device routine serves the stand-alone kernel and the combine tiles
+// of the persistent kernel.
+#pragma once
+#include "moe_dev.cuh"
+
+namespace moe {
+
+// Tokens [t0, t1) by `nthr` cooperating threads (thread index tid); 8 bf16 per 16-byte access.
+__device__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, int H, int tid,
+                                      int nthr) {
+  const int vec_per_row = H / 8;
+  const uint4* D = reinterpret_cast<const uint4*>(op->D);
+  uint4* y = reinterpret_cast<uint4*>(op->y);
+  const int* f2s = op->flat_to_sorted;
+  const float* w = op->topk_w;
+  const int total = (t1 - t0) * vec_per_row;
+  for (int idx = tid; idx < total; idx += nthr) {
+    const int t = t0 + idx / vec_per_row, v = idx % vec_per_row;
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+    for (int j = 0; j < k; ++j) {
+      const int p = f2s[(size_t)t * k + j];
+      const float wj = w[(size_t)t * k + j];
+      const uint4 d = D[(size_t)p * vec_per_row + v];
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&d);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(h[i]);
+        acc[2 * i] = fmaf(wj, f.x, acc[2 * i]);
+        acc[2 * i + 1] = fmaf(wj, f.y, acc[2 * i + 1]);
+      }
+    }
+    uint4 o;
+    __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+    y[(size_t)t * vec_per_row + v] = o;
+  }
+}
+
+}  // namespace moe

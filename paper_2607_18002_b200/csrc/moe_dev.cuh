@@ -1,0 +1,132 @@
+// Device-side data structures shared by the plan, run and combine kernels and the host
+// code that lays them out inside the caller's workspace.
+#pragma once
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/moe_apk.h"
+
+namespace moe {
+
+constexpr int kTileM = MOE_TILE_M;   // token rows per tile (M_t)
+constexpr int kTileN1 = 128;         // SwiGLU output columns per gate/up tile (256 weight rows)
+constexpr int kTileN2 = 256;         // output columns per down-GEMM tile
+constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle row of bf16)
+constexpr int kStages = 4;           // shared-memory pipeline depth
+constexpr int kCombineTokens = 32;   // tokens per combine tile
+constexpr int kPlanChunk = 256;      // routed rows ranked by one warp in the plan kernels
+constexpr int kGroupMTiles = 16;     // m-tiles per dependency group of the tile list
+constexpr int kMaxOps = 16;
+constexpr int kMaxExperts = 1024;
+
+enum TileKind : int { kGateUp = 0, kDown = 1, kCombine = 2 };
+
+// tile-list entry: bits 0..19 m-tile (or combine chunk), 20..27 n-tile, 28..29 kind
+__host__ __device__ inline int pack_tile(int kind, int n, int m) { return (kind << 28) | (n << 20) | m; }
+__host__ __device__ inline int tile_kind(int t) { return (t >> 28) & 3; }
+__host__ __device__ inline int tile_n(int t) { return (t >> 20) & 0xff; }
+__host__ __device__ inline int tile_m(int t) { return t & 0xfffff; }
+
+struct MTile {   // one row block of one expert (the unit counted by x_moe)
+  int expert, row0, rows, pad;
+};
+
+// Written by the plan kernel, read by the run kernel.
+struct PlanState {
+  int n_mtiles;       // x_moe
+  int n_gemm_tiles;   // queue entries of kind gate/up or down
+  int n_comb_tiles;   // queue entries of kind combine (follow the GEMM entries)
+  int planned;        // 1 after moe_plan
+};
+
+// Zeroed by moe_run before every launch.
+struct RunState {
+  int gemm_done;      // committed GEMM tiles
+  int tiles_done;     // committed tiles of any kind
+  int done;           // 1 when the op has fully finished
+  int pad;
+};
+
+struct __align__(128) OpDev {
+  CUtensorMap tm_x;     // [T, H]      box {64, 1}   gathered rows of the activations
+  CUtensorMap tm_a;     // [Rmax, I]   box {64, 1}   packed intermediate (rows by index)
+  CUtensorMap tm_w1;    // [E*2I, H]   box {64, 128} gate/up weights
+  CUtensorMap tm_w2;    // [E*H, I]    box {64, 128} down weights
+  int cls, n_tokens, n_rows, after_op;
+  const void* x;
+  const float* x_scale;
+  const int* topk_ids;
+  const float* topk_w;
+  const void* w_gate_up;
+  const void* w_down;
+  const float* s_gate_up;
+  const float* s_down;
+  void* y;
+  int* counts;
+  int* offsets;
+  int* sorted_to_flat;
+  int* flat_to_sorted;
+  const unsigned* ready;
+  unsigned* done;
+  // workspace-owned
+  __nv_bfloat16* A;      // [Rmax, I]  SwiGLU output, packed order
+  __nv_bfloat16* D;      // [Rmax, H]  expert output, packed order
+  MTile* mtiles;         // [max_mtiles]
+  int* tile_list;        // [max_tiles]
+  int* plan_hist;        // [n_chunks, E] per-warp histogram, then per-warp base rank
+  PlanState* plan;
+  RunState* run;
+  int* g1_done;          // [max_mtiles] committed gate/up tiles per m-tile
+};
+
+struct Status {   // first error wins (atomicCAS on code)
+  int code;
+  int detail[4];
+  int abort;      // set with code; every CTA stops claiming when it sees it
+  int pad[2];
+};
+
+struct Global {
+  Status status;
+  int budget;             // decode SM budget q (Section 5.4)
+  int pad[7];
+};
+
+// Start of the region moe_run zeroes before every launch; the per-slot RunState blocks and
+// g1_done arrays follow it.
+struct RunHead {
+  unsigned heads[2];      // next ticket of the decode / prefill queue
+  unsigned log_count;
+  int pad[5];
+};
+
+struct RunArgs {
+  Global* g;
+  OpDev* ops;             // indexed by slot
+  moe_tile_rec_t* log;
+  int log_cap;
+  int n_ops;
+  int fuse_combine;
+  int E, k, H, I;
+  long long wait_ns;
+  int slots[kMaxOps];
+};
+
+__device__ inline void report(Status* st, int code, int d0, int d1, int d2, int d3) {
+  if (atomicCAS(&st->code, 0, code) == 0) {
+    st->detail[0] = d0; st->detail[1] = d1; st->detail[2] = d2; st->detail[3] = d3;
+  }
+  __threadfence();
+  atomicExch(&st->abort, 1);
+}
+
+__device__ inline unsigned long long gtime_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+}  // namespace moe

@@ -1,0 +1,338 @@
+// Host side of the C ABI: argument validation, the layout of the caller's workspace,
+// TMA descriptors, and the launches.  No hidden host synchronisation except where the
+// header says so.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "moe_dev.cuh"
+
+namespace moe {
+cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, int E, int NT1,
+                        int NT2, cudaStream_t stream);
+cudaError_t launch_combine(const OpDev* d_op, int T, int k, int H, cudaStream_t stream);
+cudaError_t prepare_run_kernel();
+cudaError_t launch_run(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream);
+}  // namespace moe
+
+using namespace moe;
+
+namespace {
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+struct Layout {
+  size_t global_off, ops_off, runzero_off, runzero_bytes, log_off, slots_off, slot_stride;
+  // inside a slot
+  size_t A_off, D_off, mtiles_off, tiles_off, hist_off, plan_off;
+  // inside the run-zero region (after RunHead)
+  size_t rs_stride;      // RunState + g1_done[max_mtiles], per slot
+  size_t total;
+  int max_rows, max_mtiles, max_tiles, NT1, NT2;
+};
+
+int check_config(const moe_config_t* c) {
+  if (!c) return MOE_EINVAL;
+  if (c->n_experts < 1 || c->n_experts > kMaxExperts) return MOE_EINVAL;
+  if (c->top_k < 1 || c->top_k > 32 || c->top_k > c->n_experts) return MOE_EINVAL;
+  if (c->hidden < kTileN2 || c->hidden % kTileN2) return MOE_EINVAL;
+  if (c->inter < kTileN1 || c->inter % kTileN1) return MOE_EINVAL;
+  if (c->dtype != MOE_DTYPE_BF16) return MOE_EINVAL;
+  if (c->max_tokens_per_op < 1 || c->max_ops < 1 || c->max_ops > kMaxOps) return MOE_EINVAL;
+  if ((long long)c->max_tokens_per_op * c->top_k > (1 << 20) * (long long)kTileM) return MOE_EINVAL;
+  if (c->wait_limit_us < 0 || c->tile_log_entries < 0 || c->n_ctas < 0) return MOE_EINVAL;
+  return MOE_OK;
+}
+
+Layout make_layout(const moe_config_t* c) {
+  Layout L{};
+  const size_t E = c->n_experts, H = c->hidden, I = c->inter;
+  L.max_rows = c->max_tokens_per_op * c->top_k;
+  L.max_mtiles = (L.max_rows + kTileM - 1) / kTileM + c->n_experts;
+  L.NT1 = (int)(I / kTileN1);
+  L.NT2 = (int)(H / kTileN2);
+  const int max_comb = (c->max_tokens_per_op + kCombineTokens - 1) / kCombineTokens;
+  L.max_tiles = L.max_mtiles * (L.NT1 + L.NT2) + max_comb;
+  const size_t n_chunks = ((size_t)L.max_rows + kPlanChunk - 1) / kPlanChunk;
+
+  size_t off = 0;
+  L.A_off = off;       off = align_up(off + (size_t)L.max_rows * I * 2, 1024);
+  L.D_off = off;       off = align_up(off + (size_t)L.max_rows * H * 2, 1024);
+  L.mtiles_off = off;  off = align_up(off + (size_t)L.max_mtiles * sizeof(MTile), 1024);
+  L.tiles_off = off;   off = align_up(off + (size_t)L.max_tiles * 4, 1024);
+  L.hist_off = off;    off = align_up(off + n_chunks * E * 4, 1024);
+  L.plan_off = off;    off = align_up(off + sizeof(PlanState), 1024);
+  L.slot_stride = off;
+
+  size_t g = 0;
+  L.global_off = g;    g = align_up(g + sizeof(Global), 1024);
+  L.ops_off = g;       g = align_up(g + sizeof(OpDev) * c->max_ops, 1024);
+  L.runzero_off = g;
+  L.rs_stride = align_up(sizeof(RunState) + (size_t)L.max_mtiles * 4, 16);
+  L.runzero_bytes = align_up(sizeof(RunHead) + L.rs_stride * c->max_ops, 1024);
+  g += L.runzero_bytes;
+  L.log_off = g;       g = align_up(g + (size_t)c->tile_log_entries * sizeof(moe_tile_rec_t), 1024);
+  L.slots_off = g;
+  L.total = g + L.slot_stride * c->max_ops;
+  return L;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+}  // namespace
+
+struct moe_ctx {
+  moe_config_t cfg;
+  Layout L;
+  unsigned char* ws;
+  int n_ctas, sm_count;
+  EncodeTiledFn encode;
+  moe_op_t ops[kMaxOps];
+  bool planned[kMaxOps];
+  Global* g() const { return reinterpret_cast<Global*>(ws + L.global_off); }
+  RunHead* rh() const { return reinterpret_cast<RunHead*>(ws + L.runzero_off); }
+  unsigned char* slot_base(int s) const { return ws + L.slots_off + L.slot_stride * s; }
+  OpDev* op_dev(int s) const { return reinterpret_cast<OpDev*>(ws + L.ops_off) + s; }
+  unsigned char* rs_base(int s) const { return ws + L.runzero_off + sizeof(RunHead) + L.rs_stride * s; }
+};
+
+namespace {
+
+// 2-D bf16 tensor map: `rows` x `cols` row-major, box = box_rows x 64 columns, 128-byte swizzle
+int make_map(moe_ctx* ctx, CUtensorMap* out, const void* base, size_t rows, size_t cols,
+             int box_rows) {
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+                           strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? MOE_OK : MOE_ECUDA;
+}
+
+// a stream-ordered 4-byte write: the value travels in the launch, not through host memory
+__global__ void set_word_kernel(int* p, int v) { *reinterpret_cast<volatile int*>(p) = v; }
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
+
+}  // namespace
+
+extern "C" {
+
+const char* moe_strerror(int code) {
+  switch (code) {
+    case MOE_OK: return "ok";
+    case MOE_EINVAL: return "invalid argument";
+    case MOE_ENOSPC: return "workspace or slot capacity too small";
+    case MOE_ECUDA: return "CUDA call failed (is there a device?)";
+    case MOE_ETIMEOUT: return "a device-side wait ran out";
+    case MOE_EBADID: return "expert id out of range";
+    case MOE_EBOUNDS: return "device-side index check failed";
+    case MOE_ENOTPLANNED: return "slot has no plan";
+    default: return "unknown error";
+  }
+}
+
+int moe_workspace_bytes(const moe_config_t* cfg, size_t* out) {
+  if (!out) return MOE_EINVAL;
+  const int rc = check_config(cfg);
+  if (rc) return rc;
+  *out = make_layout(cfg).total;
+  return MOE_OK;
+}
+
+int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_ctx_t** out) {
+  if (!out || !dev_workspace) return MOE_EINVAL;
+  int rc = check_config(cfg);
+  if (rc) return rc;
+  if (reinterpret_cast<uintptr_t>(dev_workspace) & 1023) return MOE_EINVAL;
+  Layout L = make_layout(cfg);
+  if (bytes < L.total) return MOE_ENOSPC;
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ECUDA;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return MOE_ECUDA;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn)
+    return MOE_ECUDA;
+  if (prepare_run_kernel() != cudaSuccess) return MOE_ECUDA;
+  moe_ctx* ctx = new (std::nothrow) moe_ctx();
+  if (!ctx) return MOE_ENOSPC;
+  ctx->cfg = *cfg;
+  if (ctx->cfg.wait_limit_us == 0) ctx->cfg.wait_limit_us = 2000000;
+  ctx->L = L;
+  ctx->ws = static_cast<unsigned char*>(dev_workspace);
+  ctx->sm_count = sms;
+  ctx->n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : sms;
+  ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  memset(ctx->planned, 0, sizeof(ctx->planned));
+  // zero the control blocks (status, budget, run state, plan states)
+  cudaError_t e = cudaMemset(ctx->ws, 0, L.slots_off);
+  for (int s = 0; s < cfg->max_ops && e == cudaSuccess; ++s)
+    e = cudaMemset(ctx->slot_base(s) + L.plan_off, 0, sizeof(PlanState));
+  if (e != cudaSuccess) { delete ctx; return MOE_ECUDA; }
+  *out = ctx;
+  return MOE_OK;
+}
+
+void moe_destroy(moe_ctx_t* ctx) { delete ctx; }
+
+int moe_sm_count(moe_ctx_t* ctx) { return ctx ? ctx->sm_count : MOE_EINVAL; }
+
+int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
+  if (!ctx || !op) return MOE_EINVAL;
+  const moe_config_t& c = ctx->cfg;
+  if (slot < 0 || slot >= c.max_ops) return MOE_EINVAL;
+  if (op->cls != MOE_CLASS_DECODE && op->cls != MOE_CLASS_PREFILL) return MOE_EINVAL;
+  if (op->n_tokens < 0) return MOE_EINVAL;
+  if (op->n_tokens > c.max_tokens_per_op) return MOE_ENOSPC;
+  if (op->after_op < -1 || op->after_op >= c.max_ops || op->after_op == slot) return MOE_EINVAL;
+  if (!op->counts || !op->offsets) return MOE_EINVAL;
+  if (!op->w_gate_up || !op->w_down || !aligned16(op->w_gate_up) || !aligned16(op->w_down)) return MOE_EINVAL;
+  if (op->n_tokens > 0) {
+    if (!op->x || !op->topk_ids || !op->topk_w || !op->y || !op->sorted_to_flat || !op->flat_to_sorted)
+      return MOE_EINVAL;
+    if (!aligned16(op->x) || !aligned16(op->y)) return MOE_EINVAL;
+  }
+  const Layout& L = ctx->L;
+  unsigned char* sb = ctx->slot_base(slot);
+  OpDev h;
+  memset(&h, 0, sizeof(h));
+  h.cls = op->cls;
+  h.n_tokens = op->n_tokens;
+  h.n_rows = op->n_tokens * c.top_k;
+  h.after_op = op->after_op;
+  h.x = op->x; h.x_scale = op->x_scale; h.topk_ids = op->topk_ids; h.topk_w = op->topk_w;
+  h.w_gate_up = op->w_gate_up; h.w_down = op->w_down; h.s_gate_up = op->s_gate_up; h.s_down = op->s_down;
+  h.y = op->y; h.counts = op->counts; h.offsets = op->offsets;
+  h.sorted_to_flat = op->sorted_to_flat; h.flat_to_sorted = op->flat_to_sorted;
+  h.ready = op->ready; h.done = op->done;
+  h.A = reinterpret_cast<__nv_bfloat16*>(sb + L.A_off);
+  h.D = reinterpret_cast<__nv_bfloat16*>(sb + L.D_off);
+  h.mtiles = reinterpret_cast<MTile*>(sb + L.mtiles_off);
+  h.tile_list = reinterpret_cast<int*>(sb + L.tiles_off);
+  h.plan_hist = reinterpret_cast<int*>(sb + L.hist_off);
+  h.plan = reinterpret_cast<PlanState*>(sb + L.plan_off);
+  h.run = reinterpret_cast<RunState*>(ctx->rs_base(slot));
+  h.g1_done = reinterpret_cast<int*>(ctx->rs_base(slot) + sizeof(RunState));
+  int rc = MOE_OK;
+  if (op->n_tokens > 0) {
+    rc = make_map(ctx, &h.tm_x, op->x, (size_t)op->n_tokens, (size_t)c.hidden, 1);
+    if (!rc) rc = make_map(ctx, &h.tm_a, h.A, (size_t)L.max_rows, (size_t)c.inter, 1);
+    if (!rc) rc = make_map(ctx, &h.tm_w1, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 128);
+    if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
+    if (rc) return rc;
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemcpyAsync(ctx->op_dev(slot), &h, sizeof(h), cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return MOE_ECUDA;
+  if (launch_plan(ctx->op_dev(slot), ctx->g(), slot, op->n_tokens, c.top_k, c.n_experts, L.NT1, L.NT2,
+                  st) != cudaSuccess)
+    return MOE_ECUDA;
+  ctx->ops[slot] = *op;
+  ctx->planned[slot] = true;
+  return MOE_OK;
+}
+
+int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, void* stream) {
+  if (!ctx || !slots || n_ops < 1 || n_ops > ctx->cfg.max_ops) return MOE_EINVAL;
+  const moe_config_t& c = ctx->cfg;
+  RunArgs a;
+  memset(&a, 0, sizeof(a));
+  for (int i = 0; i < n_ops; ++i) {
+    const int s = slots[i];
+    if (s < 0 || s >= c.max_ops) return MOE_EINVAL;
+    if (!ctx->planned[s]) return MOE_ENOTPLANNED;
+    for (int j = 0; j < i; ++j) if (slots[j] == s) return MOE_EINVAL;
+    a.slots[i] = s;
+  }
+  for (int i = 0; i < n_ops; ++i) {      // after_op must name an op of this run
+    const int dep = ctx->ops[slots[i]].after_op;
+    if (dep < 0) continue;
+    bool found = false;
+    for (int j = 0; j < n_ops; ++j) found |= slots[j] == dep;
+    if (!found) return MOE_EINVAL;
+  }
+  a.g = ctx->g();
+  a.ops = ctx->op_dev(0);
+  a.log = reinterpret_cast<moe_tile_rec_t*>(ctx->ws + ctx->L.log_off);
+  a.log_cap = c.tile_log_entries;
+  a.n_ops = n_ops;
+  a.fuse_combine = fuse_combine ? 1 : 0;
+  a.E = c.n_experts; a.k = c.top_k; a.H = c.hidden; a.I = c.inter;
+  a.wait_ns = (long long)c.wait_limit_us * 1000;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
+  if (launch_run(a, ctx->rh(), ctx->n_ctas, st) != cudaSuccess) return MOE_ECUDA;
+  return MOE_OK;
+}
+
+int moe_combine(moe_ctx_t* ctx, int slot, void* stream) {
+  if (!ctx || slot < 0 || slot >= ctx->cfg.max_ops) return MOE_EINVAL;
+  if (!ctx->planned[slot]) return MOE_ENOTPLANNED;
+  if (launch_combine(ctx->op_dev(slot), ctx->ops[slot].n_tokens, ctx->cfg.top_k, ctx->cfg.hidden,
+                     static_cast<cudaStream_t>(stream)) != cudaSuccess)
+    return MOE_ECUDA;
+  return MOE_OK;
+}
+
+int moe_set_budget(moe_ctx_t* ctx, int decode_sms, void* stream) {
+  if (!ctx || decode_sms < 0) return MOE_EINVAL;
+  set_word_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(&ctx->g()->budget, decode_sms);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ECUDA;
+}
+
+int moe_status(moe_ctx_t* ctx, int32_t* code, int32_t detail[4]) {
+  if (!ctx || !code) return MOE_EINVAL;
+  Status s;
+  if (cudaMemcpy(&s, &ctx->g()->status, sizeof(s), cudaMemcpyDeviceToHost) != cudaSuccess) return MOE_ECUDA;
+  *code = s.code;
+  if (detail) for (int i = 0; i < 4; ++i) detail[i] = s.detail[i];
+  if (s.code != 0 || s.abort != 0)
+    if (cudaMemset(&ctx->g()->status, 0, sizeof(Status)) != cudaSuccess) return MOE_ECUDA;
+  return MOE_OK;
+}
+
+int moe_footprint(moe_ctx_t* ctx, int slot, int32_t* x_moe, int32_t* n_tiles) {
+  if (!ctx || slot < 0 || slot >= ctx->cfg.max_ops) return MOE_EINVAL;
+  if (!ctx->planned[slot]) return MOE_ENOTPLANNED;
+  PlanState ps;
+  if (cudaMemcpy(&ps, ctx->slot_base(slot) + ctx->L.plan_off, sizeof(ps), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return MOE_ECUDA;
+  if (x_moe) *x_moe = ps.n_mtiles;
+  if (n_tiles) *n_tiles = ps.n_gemm_tiles + ps.n_comb_tiles;
+  return MOE_OK;
+}
+
+int moe_read_tile_table(moe_ctx_t* ctx, int slot, int32_t* host_out, int max_tiles) {
+  if (!ctx || !host_out || slot < 0 || slot >= ctx->cfg.max_ops || max_tiles < 0) return MOE_EINVAL;
+  if (!ctx->planned[slot]) return MOE_ENOTPLANNED;
+  int n = max_tiles < ctx->L.max_mtiles ? max_tiles : ctx->L.max_mtiles;
+  if (n > 0 && cudaMemcpy(host_out, ctx->slot_base(slot) + ctx->L.mtiles_off, (size_t)n * sizeof(MTile),
+                          cudaMemcpyDeviceToHost) != cudaSuccess)
+    return MOE_ECUDA;
+  return MOE_OK;
+}
+
+int moe_read_tile_log(moe_ctx_t* ctx, moe_tile_rec_t* host_out, int max_records, int* n) {
+  if (!ctx || !host_out || !n || max_records < 0) return MOE_EINVAL;
+  RunHead rh;
+  if (cudaMemcpy(&rh, ctx->rh(), sizeof(rh), cudaMemcpyDeviceToHost) != cudaSuccess) return MOE_ECUDA;
+  int cnt = (int)rh.log_count;
+  if (cnt > ctx->cfg.tile_log_entries) cnt = ctx->cfg.tile_log_entries;
+  if (cnt > max_records) cnt = max_records;
+  if (cnt > 0 && cudaMemcpy(host_out, ctx->ws + ctx->L.log_off, (size_t)cnt * sizeof(moe_tile_rec_t),
+                            cudaMemcpyDeviceToHost) != cudaSuccess)
+    return MOE_ECUDA;
+  *n = cnt;
+  return MOE_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,225 @@
+// moe_plan: top-k expert ids -> per-expert counts, exclusive offsets (device prefix sum),
+// the stable permutation of routed rows, the m-tile table (its length is the footprint
+// x_moe of Section 5.2 of the paper) and the ordered tile list the persistent kernel's
+// queues serve.
+//
+// The permutation is one stable counting-sort pass over the expert id.  No atomic decides
+// an order: every warp ranks a fixed chunk of rows, a column scan over the per-warp
+// histograms gives each warp its base rank per expert, and inside a warp rows are ranked
+// by lane order, so the result is unique and reproducible.
+#include "moe_dev.cuh"
+
+namespace moe {
+
+constexpr int kPlanThreads = 256;
+constexpr int kPlanWarps = kPlanThreads / 32;
+
+// ---------------------------------------------------------------- K1: per-warp histograms
+__global__ void __launch_bounds__(kPlanThreads)
+plan_hist_kernel(const OpDev* __restrict__ op, Global* g, int slot, int R, int E) {
+  extern __shared__ int sm[];                 // [kPlanWarps][E]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x * kPlanWarps + warp;
+  int* h = sm + warp * E;
+  for (int e = lane; e < E; e += 32) h[e] = 0;
+  __syncwarp();
+  const int* ids = op->topk_ids;
+  const int base = chunk * kPlanChunk;
+  for (int it = 0; it < kPlanChunk / 32; ++it) {
+    const int i = base + it * 32 + lane;
+    int id = -1;
+    if (i < R) {
+      id = ids[i];
+      if (id < 0 || id >= E) {
+        report(&g->status, MOE_EBADID, slot, i, id, 0);
+        id = -1;
+      }
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, id);
+    if (id >= 0 && (peers & ((1u << lane) - 1)) == 0) h[id] += __popc(peers);
+    __syncwarp();
+  }
+  int* out = op->plan_hist + (size_t)chunk * E;
+  if (base < R)
+    for (int e = lane; e < E; e += 32) out[e] = h[e];
+}
+
+// exclusive scan of one int per thread over a 1024-thread block
+__device__ inline int block_excl_scan(int v, int* total, int* warp_sums) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  int inc = v;
+#pragma unroll
+  for (int d = 1; d < 32; d <<= 1) {
+    int n = __shfl_up_sync(0xffffffffu, inc, d);
+    if (lane >= d) inc += n;
+  }
+  if (lane == 31) warp_sums[warp] = inc;
+  __syncthreads();
+  if (warp == 0) {
+    int s = warp_sums[lane];
+    int si = s;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+      int n = __shfl_up_sync(0xffffffffu, si, d);
+      if (lane >= d) si += n;
+    }
+    warp_sums[lane] = si - s;               // exclusive warp offsets
+    if (lane == 31) warp_sums[32] = si;     // grand total
+  }
+  __syncthreads();
+  const int res = warp_sums[warp] + inc - v;
+  *total = warp_sums[32];
+  __syncthreads();
+  return res;
+}
+
+// ---------------------------------------------------------------- K2: scans + tile table + tile list
+__global__ void __launch_bounds__(1024)
+plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int NT1, int NT2,
+                 int T) {
+  __shared__ int warp_sums[33];
+  __shared__ int s_cnt[kMaxExperts], s_m0[kMaxExperts], s_grp[kMaxExperts], s_moff[kMaxExperts];
+  __shared__ int g_first[kMaxExperts], g_cnt[kMaxExperts], g_base1[kMaxExperts], g_base2[kMaxExperts];
+  __shared__ int s_ngroups, s_ntiles;
+  const int e = threadIdx.x;
+
+  // column scan over the per-warp histograms: base rank of every (warp chunk, expert)
+  int cnt = 0;
+  if (e < E) {
+    int* hcol = op->plan_hist + e;
+    for (int c = 0; c < n_chunks; ++c) {
+      const int v = hcol[(size_t)c * E];
+      hcol[(size_t)c * E] = cnt;
+      cnt += v;
+    }
+  }
+  int total;
+  const int off = block_excl_scan(cnt, &total, warp_sums);       // device prefix sum over experts
+  if (e < E) {
+    op->counts[e] = cnt;
+    op->offsets[e] = off;
+    int* hcol = op->plan_hist + e;
+    for (int c = 0; c < n_chunks; ++c) hcol[(size_t)c * E] += off;
+    s_cnt[e] = cnt;
+  }
+  if (e == 0) op->offsets[E] = total;
+
+  // m-tiles: ceil(m_e / M_t) per expert with rows (the footprint x_moe)
+  const int me = (e < E) ? (cnt + kTileM - 1) / kTileM : 0;
+  int x_moe;
+  const int m0 = block_excl_scan(me, &x_moe, warp_sums);
+  if (e < E) {
+    s_m0[e] = m0;
+    for (int j = 0; j < me; ++j) {
+      MTile t;
+      t.expert = e;
+      t.row0 = off + j * kTileM;
+      t.rows = min(kTileM, cnt - j * kTileM);
+      t.pad = 0;
+      op->mtiles[m0 + j] = t;
+    }
+  }
+  __syncthreads();
+
+  // dependency groups: consecutive experts holding at least kGroupMTiles m-tiles.  The
+  // list is  G1(g0) G1(g1) G2(g0) G1(g2) G2(g1) ... G2(last): every down-GEMM tile comes
+  // after all gate/up tiles of its group and of one more group, so by the time it is
+  // claimed the tiles it depends on were claimed long before.
+  if (threadIdx.x == 0) {
+    int ng = 0, acc = 0, first = 0;
+    for (int x = 0; x < E; ++x) {
+      const int m = (s_cnt[x] + kTileM - 1) / kTileM;
+      s_grp[x] = ng;
+      s_moff[x] = acc;
+      acc += m;
+      if (acc >= kGroupMTiles || x == E - 1) {
+        if (acc > 0) { g_first[ng] = first; g_cnt[ng] = acc; ++ng; }
+        else { /* trailing empty experts join nothing */ }
+        first += acc;
+        acc = 0;
+      }
+    }
+    int pos = 0;
+    for (int gi = 0; gi < ng; ++gi) {
+      g_base1[gi] = pos;
+      pos += g_cnt[gi] * NT1;
+      if (gi >= 1) { g_base2[gi - 1] = pos; pos += g_cnt[gi - 1] * NT2; }
+    }
+    if (ng > 0) { g_base2[ng - 1] = pos; pos += g_cnt[ng - 1] * NT2; }
+    s_ngroups = ng;
+    s_ntiles = pos;
+  }
+  __syncthreads();
+
+  for (int m = threadIdx.x; m < x_moe; m += blockDim.x) {
+    const int ex = op->mtiles[m].expert;
+    const int gi = s_grp[ex];
+    const int Me = (s_cnt[ex] + kTileM - 1) / kTileM;
+    const int j = m - s_m0[ex];
+    const int b1 = g_base1[gi] + s_moff[ex] * NT1, b2 = g_base2[gi] + s_moff[ex] * NT2;
+    for (int n = 0; n < NT1; ++n) op->tile_list[b1 + n * Me + j] = pack_tile(kGateUp, n, m);
+    for (int n = 0; n < NT2; ++n) op->tile_list[b2 + n * Me + j] = pack_tile(kDown, n, m);
+  }
+  const int n_gemm = s_ntiles;
+  const int n_comb = (T + kCombineTokens - 1) / kCombineTokens;
+  for (int c = threadIdx.x; c < n_comb; c += blockDim.x)
+    op->tile_list[n_gemm + c] = pack_tile(kCombine, 0, c);
+  if (threadIdx.x == 0) {
+    PlanState ps;
+    ps.n_mtiles = x_moe;
+    ps.n_gemm_tiles = n_gemm;
+    ps.n_comb_tiles = n_comb;
+    ps.planned = 1;
+    *op->plan = ps;
+  }
+}
+
+// ---------------------------------------------------------------- K3: stable scatter
+__global__ void __launch_bounds__(kPlanThreads)
+plan_scatter_kernel(const OpDev* __restrict__ op, int R, int E) {
+  extern __shared__ int sm[];                 // [kPlanWarps][E] running rank per expert
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int chunk = blockIdx.x * kPlanWarps + warp;
+  const int base = chunk * kPlanChunk;
+  if (base >= R) return;
+  int* run = sm + warp * E;
+  const int* src = op->plan_hist + (size_t)chunk * E;
+  for (int e = lane; e < E; e += 32) run[e] = src[e];
+  __syncwarp();
+  const int* ids = op->topk_ids;
+  int* s2f = op->sorted_to_flat;
+  int* f2s = op->flat_to_sorted;
+  for (int it = 0; it < kPlanChunk / 32; ++it) {
+    const int i = base + it * 32 + lane;
+    int id = -1;
+    if (i < R) {
+      id = ids[i];
+      if (id < 0 || id >= E) id = -1;       // reported by the histogram kernel
+    }
+    const unsigned peers = __match_any_sync(0xffffffffu, id);
+    const unsigned before = peers & ((1u << lane) - 1);
+    int p = -1;
+    if (id >= 0) p = run[id] + __popc(before);
+    __syncwarp();
+    if (id >= 0 && before == 0) run[id] += __popc(peers);
+    __syncwarp();
+    if (p >= 0 && p < R) {
+      s2f[p] = i;
+      f2s[i] = p;
+    }
+  }
+}
+
+cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, int E, int NT1,
+                        int NT2, cudaStream_t stream) {
+  const int R = T * k;
+  const int n_chunks = (R + kPlanChunk - 1) / kPlanChunk;
+  const int blocks = (n_chunks + kPlanWarps - 1) / kPlanWarps;
+  const size_t smem = (size_t)kPlanWarps * E * sizeof(int);
+  if (blocks > 0) plan_hist_kernel<<<blocks, kPlanThreads, smem, stream>>>(d_op, g, slot, R, E);
+  plan_scan_kernel<<<1, 1024, 0, stream>>>(d_op, n_chunks, R, E, NT1, NT2, T);
+  if (blocks > 0) plan_scatter_kernel<<<blocks, kPlanThreads, smem, stream>>>(d_op, R, E);
+  return cudaGetLastError();
+}
+
+}  // namespace moe

@@ -1,0 +1,283 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the
+same seeded inputs.  Plan outputs are compared bit-exactly, outputs within
+|gpu - ref| <= 1e-2 + 1e-2 |ref| elementwise plus a relative-L2 bound of 5e-3."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_18002_b200 as moe
+from workloads import synth
+
+from gpu_util import (assert_close, bind_ops, check_plan, check_tiles, make_ctx, oracle_weights,
+                      weights_to)
+
+pytestmark = pytest.mark.gpu
+
+SMALL = synth.Spec("small", synth.Shape(8, 2, 256, 128), ((synth.PREFILL, 300), (synth.DECODE, 37)),
+                   "softmax_topk", None, 1.0, -1.0, 21)
+
+
+def _run_spec(spec, fuse, budget=None, ops=None, W=None, **ctx_kw):
+    W = W or synth.make_weights(spec)
+    ops = ops or synth.make_ops(spec)
+    Wd = weights_to(W)
+    ctx = make_ctx(spec, max_tokens=max(o.T for o in ops), max_ops=len(ops), **ctx_kw)
+    bound = bind_ops(ctx, ops, Wd)
+    if budget is not None:
+        ctx.set_budget(budget)
+    for s, b in enumerate(bound):
+        ctx.plan(s, b)
+    ctx.run(list(range(len(bound))), fuse_combine=fuse)
+    if not fuse:
+        for s in range(len(bound)):
+            ctx.combine(s)
+    ctx.check()
+    return ctx, bound, ops, W
+
+
+# ------------------------------------------------------------------ plan (bit-exact)
+
+@pytest.mark.parametrize("name", ["c1", "c2", "c3", "c4", "c5"])
+def test_plan_bit_exact_on_every_config_routing(name):
+    spec = synth.SPECS[name]
+    # the plan does not depend on H, I or the dtype: small weights keep the test light
+    small = synth.scaled(spec, shape=synth.Shape(spec.shape.E, spec.shape.k, 256, 128))
+    Wd = weights_to(synth.make_weights(small))
+    ctx = make_ctx(small)
+    for layer in range(min(spec.layers, 2)):
+        for i, (cls, T) in enumerate(spec.ops):
+            ids, w = synth.make_routing(spec, T, layer, i)
+            op = synth.Op(cls, torch.zeros(T, 256, dtype=torch.bfloat16), ids, w)
+            b = bind_ops(ctx, [op], Wd)[0]
+            ctx.plan(i, b)
+            ctx.check()
+            counts = check_plan(b, op, spec.shape.E)
+            check_tiles(ctx, i, counts)
+
+
+@pytest.mark.parametrize("kind,T,E,k", [
+    ("one_expert", 300, 8, 2), ("two_hot", 129, 16, 2), ("round_robin", 1000, 7, 3),
+    ("random", 1, 4, 1), ("random", 127, 256, 8), ("random", 128, 256, 8), ("random", 4099, 64, 6),
+    ("round_robin", 64, 1, 1), ("round_robin", 257, 2, 2)])
+def test_plan_adversarial_routings(kind, T, E, k):
+    sh = synth.Shape(E, k, 256, 128)
+    spec = synth.Spec("adv", sh, ((synth.PREFILL, T),), "uniform", None, 1.0, -1.0, 5)
+    Wd = weights_to(synth.make_weights(spec))
+    ctx = make_ctx(spec)
+    ids = synth.adversarial_ids(kind, T, E, k)
+    op = synth.Op(synth.PREFILL, torch.zeros(T, 256, dtype=torch.bfloat16), ids,
+                  np.full(ids.shape, 1.0 / k, np.float32))
+    b = bind_ops(ctx, [op], Wd)[0]
+    ctx.plan(0, b)
+    ctx.check()
+    counts = check_plan(b, op, E)
+    check_tiles(ctx, 0, counts)
+    assert counts.sum() == T * k
+
+
+def test_plan_counts_at_tile_height_boundaries():
+    E, k = 4, 1
+    for c in (127, 128, 129, 256, 257):
+        ids = np.concatenate([np.zeros(c), np.full(5, 2)]).astype(np.int32).reshape(-1, 1)
+        sh = synth.Shape(E, k, 256, 128)
+        spec = synth.Spec("edge", sh, ((synth.PREFILL, ids.shape[0]),), "uniform", None, 1.0, -1.0, 6)
+        ctx = make_ctx(spec)
+        Wd = weights_to(synth.make_weights(spec))
+        op = synth.Op(synth.PREFILL, torch.zeros(ids.shape[0], 256, dtype=torch.bfloat16), ids,
+                      np.ones(ids.shape, np.float32))
+        b = bind_ops(ctx, [op], Wd)[0]
+        ctx.plan(0, b)
+        ctx.check()
+        counts = check_plan(b, op, E)
+        check_tiles(ctx, 0, counts)
+        assert ctx.footprint(0)[0] == -(-c // 128) + 1
+
+
+def test_bad_expert_id_is_reported_not_fatal():
+    spec = SMALL
+    ctx = make_ctx(spec)
+    Wd = weights_to(synth.make_weights(spec))
+    ops = synth.make_ops(spec)
+    ops[0].ids[5, 1] = 99
+    b = bind_ops(ctx, ops[:1], Wd)[0]
+    ctx.plan(0, b)
+    torch.cuda.synchronize()
+    code, detail = ctx.status()
+    assert code == moe.MOE_EBADID and detail[1] == 5 * 2 + 1 and detail[2] == 99
+    assert ctx.status()[0] == 0            # cleared; the context stays usable
+    ops = synth.make_ops(spec)
+    b = bind_ops(ctx, ops[:1], Wd)[0]
+    ctx.plan(0, b)
+    ctx.check()
+    check_plan(b, ops[0], spec.shape.E)
+
+
+# ------------------------------------------------------------------ the whole path
+
+@pytest.mark.parametrize("fuse", [False, True])
+@pytest.mark.parametrize("spec", [synth.SPECS["c1u"], SMALL], ids=["c1u", "small_ragged"])
+def test_small_configs_match_oracle(spec, fuse):
+    ctx, bound, ops, W = _run_spec(spec, fuse)
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        ref = oracle.forward(OW, op.x, None, op.ids, op.w)
+        check_plan(b, op, spec.shape.E)
+        assert_close(b.y.float().cpu().numpy(), ref["y"])
+
+
+def test_c1_as_stated():
+    """C1 with its stated N(0, 0.02) tensors: outputs are ~1e-5, so the absolute term of the
+    tolerance is void; the relative-L2 bound is what checks it."""
+    spec = synth.SPECS["c1"]
+    ctx, bound, ops, W = _run_spec(spec, True)
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        ref = oracle.forward(OW, op.x, None, op.ids, op.w)
+        assert_close(b.y.float().cpu().numpy(), ref["y"], rel_l2=1e-2)
+
+
+def test_one_expert_takes_everything_and_empty_op():
+    spec = synth.scaled(SMALL, ops=((synth.PREFILL, 300), (synth.DECODE, 0)))
+    ops = synth.make_ops(spec)
+    ops[0].ids[:] = synth.adversarial_ids("one_expert", 300, 8, 2)
+    ctx, bound, ops, W = _run_spec(spec, True, ops=ops)
+    ref = oracle.forward(oracle_weights(spec, W), ops[0].x, None, ops[0].ids, ops[0].w)
+    assert_close(bound[0].y.float().cpu().numpy(), ref["y"])
+    assert ctx.footprint(1) == (0, 0)
+
+
+def test_schedule_independence_bitwise():
+    """A phase switch happens only between tiles, so the output may not depend on the budget,
+    on the class split, on fusing the combine, or on the run."""
+    spec = SMALL
+    W = synth.make_weights(spec)
+    ops = synth.make_ops(spec)
+    outs = []
+    for fuse, budget, n_ctas in ((False, 0, 0), (True, 0, 0), (True, 16, 0), (True, 1000, 0),
+                                 (True, 64, 3), (True, 1, 1), (True, 0, 0)):
+        ctx, bound, _, _ = _run_spec(spec, fuse, budget=budget, ops=ops, W=W, n_ctas=n_ctas)
+        outs.append([b.y.clone() for b in bound])
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a, b)
+    # the same tokens as one op of one class
+    whole = synth.Op(synth.PREFILL, torch.cat([o.x for o in ops]),
+                     np.concatenate([o.ids for o in ops]), np.concatenate([o.w for o in ops]))
+    spec1 = synth.scaled(spec, ops=((synth.PREFILL, whole.T),))
+    ctx, bound, _, _ = _run_spec(spec1, True, ops=[whole], W=W)
+    assert torch.equal(bound[0].y, torch.cat(outs[0]))
+
+
+def test_never_ready_op_times_out_cleanly():
+    spec = SMALL
+    W = synth.make_weights(spec)
+    Wd = weights_to(W)
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec, wait_limit_us=20000)
+    never = torch.zeros(1, dtype=torch.int32, device="cuda")
+    b0 = bind_ops(ctx, ops[:1], Wd)[0]
+    b1 = bind_ops(ctx, ops[1:], Wd, ready=never)[0]
+    ctx.plan(0, b0)
+    ctx.plan(1, b1)
+    ctx.run([0, 1], fuse_combine=True)
+    torch.cuda.synchronize()
+    code, detail = ctx.status()
+    assert code == moe.MOE_ETIMEOUT and detail[0] == 1
+    # the prefill op still finished, and the context is usable afterwards
+    ref = oracle.forward(oracle_weights(spec, W), ops[0].x, None, ops[0].ids, ops[0].w)
+    assert_close(b0.y.float().cpu().numpy(), ref["y"])
+    never.fill_(1)
+    ctx.run([0, 1], fuse_combine=True)
+    ctx.check()
+    ref1 = oracle.forward(oracle_weights(spec, W), ops[1].x, None, ops[1].ids, ops[1].w)
+    assert_close(b1.y.float().cpu().numpy(), ref1["y"])
+
+
+def test_after_op_and_done_word():
+    spec = SMALL
+    W = synth.make_weights(spec)
+    Wd = weights_to(W)
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec, tile_log_entries=4096)
+    done = torch.zeros(2, dtype=torch.int32, device="cuda")
+    b0 = bind_ops(ctx, ops[:1], Wd, done=done[0:1])[0]
+    b1 = bind_ops(ctx, ops[1:], Wd, done=done[1:2], after_op=0)[0]
+    ctx.plan(0, b0)
+    ctx.plan(1, b1)
+    ctx.run([0, 1], fuse_combine=True)
+    ctx.check()
+    assert done.tolist() == [1, 1]
+    log = ctx.tile_log()
+    n0, n1 = ctx.footprint(0)[1], ctx.footprint(1)[1]
+    assert len(log) == n0 + n1
+    for s, n in ((0, n0), (1, n1)):                       # every tile exactly once
+        assert sorted(log["tile"][log["slot"] == s].tolist()) == list(range(n))
+    # the decode op was chained after the prefill op: none of its tiles was claimed earlier
+    assert log["t_claim"][log["slot"] == 1].min() >= log["t_commit"][log["slot"] == 0].max()
+    assert np.all(log["t_commit"] >= log["t_claim"])
+
+
+# ------------------------------------------------------------------ full-size configs
+
+@pytest.fixture(scope="module")
+def big_weights():
+    spec = synth.SPECS["c3"]
+    W = synth.make_weights(spec)
+    return spec, W, weights_to(W)
+
+
+def _sample_tokens(op, E, n_extra, seed):
+    """All edge rows (first and last row of every expert segment) plus a seeded sample."""
+    counts, offsets, s2f, f2s = oracle.plan(op.ids, E)
+    k = op.ids.shape[1]
+    edge = [s2f[offsets[e]] // k for e in range(E) if counts[e]] + \
+           [s2f[offsets[e + 1] - 1] // k for e in range(E) if counts[e]]
+    rng = np.random.default_rng(seed)
+    extra = rng.choice(op.T, size=min(n_extra, op.T), replace=False)
+    return np.unique(np.concatenate([np.array(edge, dtype=np.int64), extra])).astype(np.int32)
+
+
+def test_c2_decode_only_full(big_weights):
+    _, W, Wd = big_weights
+    spec = synth.SPECS["c2"]
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec)
+    b = bind_ops(ctx, ops, Wd)[0]
+    ctx.plan(0, b)
+    ctx.run([0], fuse_combine=True)
+    ctx.check()
+    counts = check_plan(b, ops[0], spec.shape.E)
+    check_tiles(ctx, 0, counts)
+    ref = oracle.forward(oracle_weights(spec, W), ops[0].x, None, ops[0].ids, ops[0].w)
+    assert_close(b.y.float().cpu().numpy(), ref["y"])
+
+
+@pytest.mark.parametrize("name,fuse", [("c3", True), ("c4", True), ("c4", False)])
+def test_full_size_sampled(big_weights, name, fuse):
+    """C3 / one C4 layer in the launch configuration the bench times; the oracle evaluates
+    every decode token, the rows at every expert-segment edge and a seeded token sample."""
+    _, W, Wd = big_weights
+    spec = synth.SPECS[name]
+    ops = synth.make_ops(spec, layer=1)
+    ctx = make_ctx(spec)
+    bound = bind_ops(ctx, ops, Wd)
+    ctx.set_budget(32)
+    for s, b in enumerate(bound):
+        ctx.plan(s, b)
+    ctx.run(list(range(len(bound))), fuse_combine=fuse)
+    if not fuse:
+        for s in range(len(bound)):
+            ctx.combine(s)
+    ctx.check()
+    OW = oracle_weights(spec, W)
+    for s, (b, op) in enumerate(zip(bound, ops)):
+        counts = check_plan(b, op, spec.shape.E)
+        check_tiles(ctx, s, counts)
+        toks = np.arange(op.T, dtype=np.int32) if op.cls == synth.DECODE and op.T <= 256 \
+            else _sample_tokens(op, spec.shape.E, 128, 11)
+        toks = toks[:700]
+        ref = oracle.forward_tokens(OW, op.x, None, op.ids, op.w, toks)
+        got = b.y[torch.from_numpy(toks).long().cuda()].float().cpu().numpy()
+        assert_close(got, ref)
+        assert torch.isfinite(b.y.float()).all()
