@@ -1,0 +1,374 @@
+#!/usr/bin/env python
+"""Benchmark of the routed-MoE expert hot path on B200.
+
+A "step" is one pass of the whole path -- moe_plan (counts, offsets, permutation, tile list)
+and moe_run (the persistent kernel: gate/up GEMM + SwiGLU, down GEMM, combine) -- over one
+synthetic batch of the chosen workload (for c4: all 8 layers, with moe_set_budget between
+them).  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload c2|c3|c4] [--impl reference]
+
+N > 1 runs N independent replicas (one process per GPU, no data-path collective); the
+reported value is all ranks' work over the slowest rank's device time.
+`--impl reference` times the CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from workloads import synth  # noqa: E402
+
+METRIC = "moe_expert_tflops"
+UNIT = "TFLOP/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+KERNELS_PER_PLAN = 3          # histogram, scan + tile list, scatter
+DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3)}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {k: float(p[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+    REASONS = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+               0x4: "sw_power_cap"}
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._thread = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self._nv = pynvml
+            self._h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self._h, pynvml.NVML_CLOCK_SM))
+            self._period = period_s
+        except Exception:
+            self._nv = None
+
+    def _loop(self):
+        nv = self._nv
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mask = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
+                for bit, name in self.REASONS.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop.wait(self._period)
+
+    def __enter__(self):
+        if self._nv is not None:
+            self._thread = threading.Thread(target=self._loop, daemon=True)
+            self._thread.start()
+        return self
+
+    def __exit__(self, *exc):
+        self._stop.set()
+        if self._thread is not None:
+            self._thread.join(timeout=2)
+
+    def summary(self):
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# ------------------------------------------------------------------ workloads
+
+def visible_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+class Workload:
+    """Device-resident inputs of one workload plus the calls of one step."""
+
+    def __init__(self, name: str, rank: int, device: torch.device, tile_log: int = 0):
+        import paper_2607_18002_b200 as moe
+        self.moe = moe
+        self.name = name
+        base = synth.SPECS[name]
+        self.spec = synth.scaled(base, seed=base.seed + 100 * rank)
+        sh = self.spec.shape
+        self.sh = sh
+        self.device = device
+        n_sets = 2 if self.spec.layers > 1 else 1          # c4 alternates two weight sets
+        threads = os.cpu_count() or 8
+        self.W_host = [synth.make_weights(self.spec, layer=i, threads=threads) for i in range(n_sets)]
+        self.W = [synth.Weights(w.w_gate_up.to(device), w.w_down.to(device)) for w in self.W_host]
+        self.layers = []
+        self.ctx = moe.Context(sh.E, sh.k, sh.H, sh.I, max(T for _, T in self.spec.ops),
+                               max_ops=len(self.spec.ops), tile_log_entries=tile_log,
+                               device=device)
+        self.flops = 0.0
+        self.bytes_alg = 0.0
+        self.h2d = self.d2h = 0
+        for layer in range(self.spec.layers):
+            ops = synth.make_ops(self.spec, layer)
+            W = self.W[layer % n_sets]
+            bound, host = [], []
+            active = np.zeros(sh.E, dtype=bool)
+            for op in ops:
+                hx = op.x.pin_memory()
+                hi = torch.from_numpy(op.ids).pin_memory()
+                hw = torch.from_numpy(op.w).pin_memory()
+                dx, di, dw = hx.to(device), hi.to(device), hw.to(device)
+                b = self.ctx.bind(op.cls, dx, di, dw, W.w_gate_up, W.w_down)
+                hy = torch.empty(b.y.shape, dtype=b.y.dtype).pin_memory()
+                bound.append(b)
+                host.append((hx, hi, hw, hy))
+                active[np.unique(op.ids)] = True
+                self.flops += 6.0 * op.ids.size * sh.H * sh.I
+                self.bytes_alg += 2 * op.T * sh.H * 2            # X once, y once
+                self.h2d += hx.numel() * 2 + hi.numel() * 4 + hw.numel() * 4
+                self.d2h += hy.numel() * 2
+            # weights of the union of active experts of the launch, once
+            self.bytes_alg += float(active.sum()) * 3 * sh.H * sh.I * 2
+            self.layers.append((ops, bound, host))
+        self.launches_per_step = sum(len(b) * KERNELS_PER_PLAN + 1 + (1 if self.spec.layers > 1 else 0)
+                                     for _, b, _ in self.layers)
+
+    def step(self, ev=None):
+        """Whole hot path for one batch; ev (optional) collects (before_run, after_run) events."""
+        ctx = self.ctx
+        for li, (_, bound, _) in enumerate(self.layers):
+            if self.spec.layers > 1:
+                ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
+            for s, b in enumerate(bound):
+                ctx.plan(s, b)
+            if ev is not None:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+            ctx.run(list(range(len(bound))), fuse_combine=True)
+            if ev is not None:
+                e1.record()
+                ev.append((e0, e1))
+
+    def step_e2e(self):
+        """The same step with host buffers: inputs come from pinned host memory and the
+        result goes back to it, all inside the timed region."""
+        ctx = self.ctx
+        for li, (_, bound, host) in enumerate(self.layers):
+            if self.spec.layers > 1:
+                ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
+            for s, (b, (hx, hi, hw, hy)) in enumerate(zip(bound, host)):
+                b.x.copy_(hx, non_blocking=True)
+                b.topk_ids.copy_(hi, non_blocking=True)
+                b.topk_w.copy_(hw, non_blocking=True)
+                ctx.plan(s, b)
+            ctx.run(list(range(len(bound))), fuse_combine=True)
+            for b, (_, _, _, hy) in zip(bound, host):
+                hy.copy_(b.y, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+
+
+def oracle_sample(w: Workload, seconds_target: float = 12.0):
+    """Times the CPU oracle, as it stands, on a bounded token sample of the workload's first
+    op.  Returns (TFLOP/s, cores, description)."""
+    import oracle
+    sh = w.sh
+    ops, _, _ = w.layers[0]
+    op = max(ops, key=lambda o: o.T)
+    Wh = w.W_host[0]
+    OW = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wh.w_gate_up, Wh.w_down)
+    cores = oracle.threads()
+    n, spent, done_tokens = max(2, cores // sh.k), 0.0, 0
+    rng = np.random.default_rng(0)
+    while True:                       # grow the sample until the time budget is used
+        toks = rng.choice(op.T, size=min(n, op.T), replace=False).astype(np.int32)
+        t0 = time.perf_counter()
+        oracle.plan(op.ids, sh.E)
+        oracle.forward_tokens(OW, op.x, None, op.ids, op.w, toks)
+        dt = time.perf_counter() - t0
+        spent += dt
+        done_tokens, last_dt = len(toks), dt
+        if spent + 3 * dt > seconds_target or len(toks) == op.T:
+            break
+        n *= 2
+    tflops = 6.0 * done_tokens * sh.k * sh.H * sh.I / last_dt / 1e12
+    return tflops, cores, (f"oracle plan on all {op.T} tokens + FFN/combine on {done_tokens} "
+                           f"seeded tokens of {w.name} ({last_dt:.2f} s)")
+
+
+# ------------------------------------------------------------------ arms
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the host cores, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    spec = synth.SPECS[args.workload]
+    sh = spec.shape
+    Wh = synth.make_weights(spec, threads=os.cpu_count() or 8)
+    op = max(synth.make_ops(spec), key=lambda o: o.T)
+    OW = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wh.w_gate_up, Wh.w_down)
+    cores = oracle.threads()
+    n_tok = max(4, (2 * cores) // sh.k)
+    rng = np.random.default_rng(0)
+    times = []
+    for i in range(args.warmup + args.steps):
+        toks = rng.choice(op.T, size=min(n_tok, op.T), replace=False).astype(np.int32)
+        t0 = time.perf_counter()
+        oracle.plan(op.ids, sh.E)
+        oracle.forward_tokens(OW, op.x, None, op.ids, op.w, toks)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            times.append(dt)
+    ms = 1e3 * float(np.mean(times))
+    value = 6.0 * min(n_tok, op.T) * sh.k * sh.H * sh.I / (ms / 1e3) / 1e12
+    sample = f"per step: oracle plan on all {op.T} tokens + FFN/combine on {min(n_tok, op.T)} seeded tokens"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": args.workload, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def run_ours(args):
+    from paper_2607_18002_b200 import dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
+    rank, world, local = dist.init_from_env()
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    peaks, peak_src = load_peaks()
+    w = Workload(args.workload, rank, device)
+    K, Wm = args.steps, args.warmup
+
+    for _ in range(Wm):
+        w.step()
+    w.ctx.check()
+
+    # ---- device-resident timing
+    ev = []
+    dist.barrier()
+    torch.cuda.synchronize()
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    with ClockSampler(visible_index(local)) as clk:
+        start.record()
+        for _ in range(K):
+            w.step(ev)
+        stop.record()
+        torch.cuda.synchronize()
+    dist.barrier()
+    w.ctx.check()
+    secs = start.elapsed_time(stop) / 1e3
+    run_ms = [a.elapsed_time(b) for a, b in ev]
+    value = dist.job_throughput(w.flops * K, secs) / 1e12
+    ms_per_step = 1e3 * dist.reduce_scalar(secs, "max") / K
+
+    # ---- end to end with host buffers
+    for _ in range(min(Wm, 3)):
+        w.step_e2e()
+    dist.barrier()
+    torch.cuda.synchronize()
+    s2, t2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s2.record()
+    for _ in range(K):
+        w.step_e2e()
+    t2.record()
+    torch.cuda.synchronize()
+    dist.barrier()
+    w.ctx.check()
+    e2e_value = dist.job_throughput(w.flops * K, s2.elapsed_time(t2) / 1e3) / 1e12
+
+    # ---- roofline of the dominant kernel (the persistent kernel), from live CUDA events
+    launches = len(run_ms)
+    t_run = float(np.mean(run_ms)) / 1e3
+    flops_launch = w.flops / len(w.layers)
+    bytes_launch = w.bytes_alg / len(w.layers)
+    tensor_frac = flops_launch / t_run / 1e12 / peaks["bf16_tflops"]
+    hbm_frac = bytes_launch / t_run / 1e9 / peaks["hbm_gbs"]
+    if args.workload == "c2":
+        roof = {"bound": "hbm", "achieved": bytes_launch / t_run / 1e9, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": hbm_frac}
+    else:
+        roof = {"bound": "tensor", "achieved": flops_launch / t_run / 1e12,
+                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tensor_frac}
+    roof.update({"traffic": None, "kernel": "moe_apk_kernel", "peak_source": peak_src,
+                 "launch_ms_mean": 1e3 * t_run, "launch_ms_min": float(np.min(run_ms)),
+                 "algorithmic_flops_per_launch": flops_launch,
+                 "algorithmic_bytes_per_launch": bytes_launch,
+                 "tensor_frac_of_burst": tensor_frac,
+                 "tensor_frac_of_sustained": flops_launch / t_run / 1e12 / peaks["bf16_tflops_sustained"],
+                 "hbm_frac": hbm_frac})
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, cores, sample = oracle_sample(w)
+        cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
+
+    if rank == 0:
+        sh = w.sh
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+            "warmup": Wm, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": args.workload, "ops": [[c, t] for c, t in w.spec.ops],
+                       "layers": w.spec.layers, "experts": sh.E, "top_k": sh.k, "hidden": sh.H,
+                       "inter": sh.I, "l2": "inputs_exceed_l2 (weights >> 126 MB, no flush)",
+                       "replicas": world, "fused_combine": True},
+            "clocks": clk.summary(),
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": w.h2d,
+                    "d2h_bytes_per_step": w.d2h},
+            "gpu_launches": w.launches_per_step * K,
+            "roofline": roof, "cpu_baseline": cpu}))
+    dist.shutdown()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    ds, dw = DEFAULT_STEPS[args.workload]
+    if args.impl == "reference":
+        ds, dw = 3, 1
+    args.steps = ds if args.steps is None else args.steps
+    args.warmup = max(3 if args.impl == "ours" else 0, dw if args.warmup is None else args.warmup)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -187,6 +187,7 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
   OpDev* op = &a->ops[ti.slot];
   __threadfence();
   fence_async_proxy();
+  const unsigned long long t_commit = a->log_cap > 0 ? gtime_ns() : 0ull;   // before it is published
   if (ti.kind == kGateUp) atomicAdd(&op->g1_done[ti.m], 1);
   if (ti.kind != kCombine) atomicAdd(&op->run->gemm_done, 1);
   const int done = atomicAdd(&op->run->tiles_done, 1) + 1;
@@ -200,7 +201,7 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
     if (idx < (unsigned)a->log_cap) {
       moe_tile_rec_t r;
       r.t_claim = ti.t_claim;
-      r.t_commit = gtime_ns();
+      r.t_commit = t_commit;
       r.slot = ti.slot;
       r.tile = ti.tile;
       r.cls = (int16_t)ti.cls;
