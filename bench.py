@@ -33,7 +33,7 @@ METRIC = "moe_expert_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 KERNELS_PER_PLAN = 3          # histogram, scan + tile list, scatter
-DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3)}
+DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c2s": (20, 3), "c3s": (10, 3)}
 
 
 def load_peaks():
@@ -219,6 +219,46 @@ def oracle_sample(w: Workload, seconds_target: float = 12.0):
                            f"seeded tokens of {w.name} ({last_dt:.2f} s)")
 
 
+def tile_stats(w: Workload):
+    """Per-tile service times (claim -> commit) of the last launch of one extra step, from the
+    kernel's tile log: the analogue of the paper's preemption-interval measurement."""
+    w.step()
+    w.ctx.check()
+    log = w.ctx.tile_log()
+    if len(log) == 0:
+        return None
+    if os.environ.get("MOE_BENCH_DUMP_LOG"):
+        np.save(os.environ["MOE_BENCH_DUMP_LOG"], log)
+    out = {"records": int(len(log))}
+    t0 = int(log["t_claim"].min())
+    span = (int(log["t_commit"].max()) - t0) / 1e3
+    out["kernel_span_us"] = span
+    service = (log["t_commit"].astype(np.int64) - log["t_claim"].astype(np.int64)) / 1e3
+    names = {0: "gate_up", 1: "down", 2: "combine"}
+    for cls, cname in ((0, "decode"), (1, "prefill")):
+        for kind, kname in names.items():
+            m = (log["cls"] == cls) & (log["kind"] == kind)
+            if m.any():
+                v = service[m]
+                out[f"{cname}_{kname}"] = {"n": int(m.sum()), "p50_us": float(np.percentile(v, 50)),
+                                           "p99_us": float(np.percentile(v, 99)),
+                                           "max_us": float(v.max()), "mean_us": float(v.mean())}
+    n_cta = int(log["cta"].max()) + 1
+    out["occupancy"] = float(service.sum() / (n_cta * span)) if span > 0 else None
+    # idle time between a CTA's consecutive tiles (commit -> next claim)
+    gaps = []
+    for c in range(n_cta):
+        r = log[log["cta"] == c]
+        r = r[np.argsort(r["t_claim"])]
+        if len(r) > 1:
+            gaps.append((r["t_claim"][1:].astype(np.int64) - r["t_commit"][:-1].astype(np.int64)) / 1e3)
+    if gaps:
+        g = np.concatenate(gaps)
+        out["gap_us"] = {"p50": float(np.percentile(g, 50)), "p99": float(np.percentile(g, 99)),
+                         "mean": float(g.mean())}
+    return out
+
+
 # ------------------------------------------------------------------ arms
 
 def run_reference(args):
@@ -266,7 +306,7 @@ def run_ours(args):
     device = torch.device("cuda", local)
     torch.cuda.set_device(device)
     peaks, peak_src = load_peaks()
-    w = Workload(args.workload, rank, device)
+    w = Workload(args.workload, rank, device, tile_log=(1 << 17) if args.tile_log else 0)
     K, Wm = args.steps, args.warmup
 
     for _ in range(Wm):
@@ -327,6 +367,8 @@ def run_ours(args):
                  "tensor_frac_of_sustained": flops_launch / t_run / 1e12 / peaks["bf16_tflops_sustained"],
                  "hbm_frac": hbm_frac})
 
+    tiles = tile_stats(w) if args.tile_log else None
+
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         v, cores, sample = oracle_sample(w)
@@ -346,7 +388,7 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": w.h2d,
                     "d2h_bytes_per_step": w.d2h},
             "gpu_launches": w.launches_per_step * K,
-            "roofline": roof, "cpu_baseline": cpu}))
+            "roofline": roof, "cpu_baseline": cpu, **({"tiles": tiles} if tiles else {})}))
     dist.shutdown()
 
 
@@ -355,9 +397,10 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c2s", "c3s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tile-log", action="store_true", help="add per-tile timing statistics of one extra untimed step")
     args = ap.parse_args()
     ds, dw = DEFAULT_STEPS[args.workload]
     if args.impl == "reference":

@@ -24,11 +24,14 @@ constexpr int kMaxExperts = 1024;
 
 enum TileKind : int { kGateUp = 0, kDown = 1, kCombine = 2 };
 
-// tile-list entry: bits 0..19 m-tile (or combine chunk), 20..27 n-tile, 28..29 kind
-__host__ __device__ inline int pack_tile(int kind, int n, int m) { return (kind << 28) | (n << 20) | m; }
-__host__ __device__ inline int tile_kind(int t) { return (t >> 28) & 3; }
-__host__ __device__ inline int tile_n(int t) { return (t >> 20) & 0xff; }
-__host__ __device__ inline int tile_m(int t) { return t & 0xfffff; }
+// Queue entry (16 bytes, one load per claim): x = kind | n-tile << 4 | m-tile << 12,
+// y = first packed row (first token for a combine tile), z = valid rows, w = expert.
+__host__ __device__ inline int4 make_entry(int kind, int n, int m, int row0, int rows, int expert) {
+  return make_int4(kind | (n << 4) | (m << 12), row0, rows, expert);
+}
+__host__ __device__ inline int entry_kind(const int4& e) { return e.x & 15; }
+__host__ __device__ inline int entry_n(const int4& e) { return (e.x >> 4) & 0xff; }
+__host__ __device__ inline int entry_m(const int4& e) { return (e.x >> 12) & 0xfffff; }
 
 struct MTile {   // one row block of one expert (the unit counted by x_moe)
   int expert, row0, rows, pad;
@@ -51,10 +54,11 @@ struct RunState {
 };
 
 struct __align__(128) OpDev {
-  CUtensorMap tm_x;     // [T, H]      box {64, 1}   gathered rows of the activations
-  CUtensorMap tm_a;     // [Rmax, I]   box {64, 1}   packed intermediate (rows by index)
+  CUtensorMap tm_a8;    // [Rmax, I]   box {64, 8}   packed intermediate, 8 consecutive rows
+  CUtensorMap tm_a32;   // [Rmax, I]   box {64, 32}
   CUtensorMap tm_w1;    // [E*2I, H]   box {64, 128} gate/up weights
   CUtensorMap tm_w2;    // [E*H, I]    box {64, 128} down weights
+  CUtensorMap tm_a128;  // [Rmax, I]   box {64, 128}
   int cls, n_tokens, n_rows, after_op;
   const void* x;
   const float* x_scale;
@@ -75,7 +79,7 @@ struct __align__(128) OpDev {
   __nv_bfloat16* A;      // [Rmax, I]  SwiGLU output, packed order
   __nv_bfloat16* D;      // [Rmax, H]  expert output, packed order
   MTile* mtiles;         // [max_mtiles]
-  int* tile_list;        // [max_tiles]
+  int4* tile_list;       // [max_tiles] queue entries in claim order
   int* plan_hist;        // [n_chunks, E] per-warp histogram, then per-warp base rank
   PlanState* plan;
   RunState* run;

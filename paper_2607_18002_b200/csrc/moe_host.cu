@@ -60,7 +60,7 @@ Layout make_layout(const moe_config_t* c) {
   L.A_off = off;       off = align_up(off + (size_t)L.max_rows * I * 2, 1024);
   L.D_off = off;       off = align_up(off + (size_t)L.max_rows * H * 2, 1024);
   L.mtiles_off = off;  off = align_up(off + (size_t)L.max_mtiles * sizeof(MTile), 1024);
-  L.tiles_off = off;   off = align_up(off + (size_t)L.max_tiles * 4, 1024);
+  L.tiles_off = off;   off = align_up(off + (size_t)L.max_tiles * sizeof(int4), 1024);
   L.hist_off = off;    off = align_up(off + n_chunks * E * 4, 1024);
   L.plan_off = off;    off = align_up(off + sizeof(PlanState), 1024);
   L.slot_stride = off;
@@ -217,15 +217,16 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   h.A = reinterpret_cast<__nv_bfloat16*>(sb + L.A_off);
   h.D = reinterpret_cast<__nv_bfloat16*>(sb + L.D_off);
   h.mtiles = reinterpret_cast<MTile*>(sb + L.mtiles_off);
-  h.tile_list = reinterpret_cast<int*>(sb + L.tiles_off);
+  h.tile_list = reinterpret_cast<int4*>(sb + L.tiles_off);
   h.plan_hist = reinterpret_cast<int*>(sb + L.hist_off);
   h.plan = reinterpret_cast<PlanState*>(sb + L.plan_off);
   h.run = reinterpret_cast<RunState*>(ctx->rs_base(slot));
   h.g1_done = reinterpret_cast<int*>(ctx->rs_base(slot) + sizeof(RunState));
   int rc = MOE_OK;
   if (op->n_tokens > 0) {
-    rc = make_map(ctx, &h.tm_x, op->x, (size_t)op->n_tokens, (size_t)c.hidden, 1);
-    if (!rc) rc = make_map(ctx, &h.tm_a, h.A, (size_t)L.max_rows, (size_t)c.inter, 1);
+    rc = make_map(ctx, &h.tm_a8, h.A, (size_t)L.max_rows, (size_t)c.inter, 8);
+    if (!rc) rc = make_map(ctx, &h.tm_a32, h.A, (size_t)L.max_rows, (size_t)c.inter, 32);
+    if (!rc) rc = make_map(ctx, &h.tm_a128, h.A, (size_t)L.max_rows, (size_t)c.inter, 128);
     if (!rc) rc = make_map(ctx, &h.tm_w1, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 128);
     if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
     if (rc) return rc;

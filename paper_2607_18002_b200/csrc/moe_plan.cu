@@ -152,18 +152,19 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   __syncthreads();
 
   for (int m = threadIdx.x; m < x_moe; m += blockDim.x) {
-    const int ex = op->mtiles[m].expert;
+    const MTile mt = op->mtiles[m];
+    const int ex = mt.expert;
     const int gi = s_grp[ex];
     const int Me = (s_cnt[ex] + kTileM - 1) / kTileM;
     const int j = m - s_m0[ex];
     const int b1 = g_base1[gi] + s_moff[ex] * NT1, b2 = g_base2[gi] + s_moff[ex] * NT2;
-    for (int n = 0; n < NT1; ++n) op->tile_list[b1 + n * Me + j] = pack_tile(kGateUp, n, m);
-    for (int n = 0; n < NT2; ++n) op->tile_list[b2 + n * Me + j] = pack_tile(kDown, n, m);
+    for (int n = 0; n < NT1; ++n) op->tile_list[b1 + n * Me + j] = make_entry(kGateUp, n, m, mt.row0, mt.rows, ex);
+    for (int n = 0; n < NT2; ++n) op->tile_list[b2 + n * Me + j] = make_entry(kDown, n, m, mt.row0, mt.rows, ex);
   }
   const int n_gemm = s_ntiles;
   const int n_comb = (T + kCombineTokens - 1) / kCombineTokens;
   for (int c = threadIdx.x; c < n_comb; c += blockDim.x)
-    op->tile_list[n_gemm + c] = pack_tile(kCombine, 0, c);
+    op->tile_list[n_gemm + c] = make_entry(kCombine, 0, c, c * kCombineTokens, min(kCombineTokens, T - c * kCombineTokens), 0);
   if (threadIdx.x == 0) {
     PlanState ps;
     ps.n_mtiles = x_moe;

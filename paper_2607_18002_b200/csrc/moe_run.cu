@@ -1,19 +1,22 @@
 // moe_run: the persistent expert kernel (the adaptive persistent kernel of Section 4 of the
 // paper, rebuilt for sm_100a).
 //
-// One CTA per SM, 6 warps with fixed roles:
+// One CTA per SM, 10 warps with fixed roles:
 //   warp 0     scheduler + producer.  At every tile boundary it reads the decode budget
 //              word and the two queue heads, claims the next tile (decode first for CTAs
 //              below the budget, prefill first for the others, each falling back to the
 //              other class: Sections 4.2 and 5.4), hands the tile to the other warps
 //              through a shared-memory ring guarded by mbarriers (the hand-off of
 //              Section 4.3: the first pipeline warp decides, later warps follow), waits for
-//              the tile's dependencies, then feeds the pipeline: weight tiles by tiled TMA,
-//              activation rows by TMA gather4 through the permutation.
+//              the tile's dependencies, then feeds the pipeline: weight tiles (and the
+//              packed intermediate rows of a down tile) by tiled TMA.
 //   warp 1     issues tcgen05.mma (128 x 256 x 16, bf16 -> fp32) into one of two TMEM
 //              accumulators; tcgen05.commit releases pipeline stages and publishes the
 //              accumulator.
-//   warps 2-5  epilogue: tcgen05.ld, SwiGLU (gate/up tiles), bf16 stores, then the release
+//   warps 2-5  gather: the activation rows of a gate/up tile are scattered tokens; they are
+//              copied through the permutation with 16-byte cp.async into the swizzled
+//              layout the tensor core reads.
+//   warps 6-9  epilogue: tcgen05.ld, SwiGLU (gate/up tiles), bf16 stores, then the release
 //              of dependency counters, the op's done word and the tile log.  They also run
 //              the combine tiles.
 // A phase switch happens only between tiles, so no accumulator, TMA transaction or buffer is
@@ -26,7 +29,8 @@
 
 namespace moe {
 
-constexpr int kThreads = 192;
+constexpr int kGatherThreads = 128;                     // 4 gather warps
+constexpr int kThreads = 64 + kGatherThreads + 128;     // scheduler/TMA, MMA, gather x4, epilogue x4
 constexpr int kABytes = kTileM * kBlockK * 2;          // 16 KB activations per stage
 constexpr int kBHalfBytes = 128 * kBlockK * 2;         // 16 KB per 128 weight rows
 constexpr int kBBytes = 2 * kBHalfBytes;               // 32 KB weights per stage
@@ -41,7 +45,7 @@ struct TileInfo {
 };
 
 struct SharedCtl {
-  unsigned long long full[kStages], empty[kStages];
+  unsigned long long full[kStages], fullA[kStages], empty[kStages];
   unsigned long long tfull[2], tempty[2];
   unsigned long long ifull[kRing], iempty[kRing];
   TileInfo info[kRing];
@@ -112,67 +116,98 @@ __device__ inline bool op_ready(const RunArgs* a, const OpDev* op) {
   return true;
 }
 
-// 1: claimed (ti filled), 0: queue exhausted, -1: head op not ready
-__device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, int cls, TileInfo& ti) {
+// Claim by the whole producer warp.  1: claimed (ti filled), 0: queue exhausted, -1: the op
+// at the head of the queue is not ready.  The head is only peeked before the fetch-add, so no
+// CTA can be starved by others (a compare-and-swap loop starves the SMs far from the counter);
+// the price is that a ticket can land just past an op boundary, in an op that is not ready
+// yet -- the caller then waits for it (bounded), holding only tickets whose predecessors in
+// the queue are all claimed already.
+__device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, int cls, int lane,
+                                TileInfo& ti, bool& need_ready) {
   const int n = sc->n_cls[cls];
   if (n == 0) return 0;
   const unsigned total = sc->cum[cls][n];
-  unsigned h = *reinterpret_cast<volatile unsigned*>(&rh->heads[cls]);
-  while (true) {
-    if (h >= total) return 0;
-    int i = 0;
-    while (h >= sc->cum[cls][i + 1]) ++i;
-    const int slot = sc->cls_slot[cls][i];
-    const OpDev* op = &a->ops[slot];
-    if (!op_ready(a, op)) return -1;
-    const unsigned old = atomicCAS(&rh->heads[cls], h, h + 1);
-    if (old == h) {
-      const int local = (int)(h - sc->cum[cls][i]);
-      const int entry = op->tile_list[local];
-      ti.kind = tile_kind(entry);
-      ti.slot = slot;
-      ti.tile = local;
-      ti.m = tile_m(entry);
-      ti.n = tile_n(entry);
-      ti.cls = cls;
-      if (ti.kind == kCombine) {
-        ti.row0 = ti.m * kCombineTokens;
-        ti.rows = min(kCombineTokens, op->n_tokens - ti.row0);
-        ti.expert = 0;
-        ti.kblocks = 0;
-      } else {
-        const MTile mt = op->mtiles[ti.m];
-        ti.row0 = mt.row0;
-        ti.rows = mt.rows;
-        ti.expert = mt.expert;
-        ti.kblocks = (ti.kind == kGateUp ? a->H : a->I) / kBlockK;
-      }
-      return 1;
-    }
-    h = old;
+  const unsigned h = *reinterpret_cast<volatile unsigned*>(&rh->heads[cls]);
+  if (h >= total) return 0;
+  int i = 0;
+  while (h >= sc->cum[cls][i + 1]) ++i;
+  int slot = sc->cls_slot[cls][i];
+  const OpDev* op = &a->ops[slot];
+  if (!op_ready(a, op)) return -1;
+  // the 32 entries from the head on are fetched while the fetch-add is in flight
+  const unsigned base = h - sc->cum[cls][i];
+  const unsigned n_op = sc->cum[cls][i + 1] - sc->cum[cls][i];
+  int4 e = make_int4(0, 0, 0, 0);
+  if (base + lane < n_op) e = op->tile_list[base + lane];
+  unsigned t = 0;
+  if (lane == 0) t = atomicAdd(&rh->heads[cls], 1u);
+  t = __shfl_sync(0xffffffffu, t, 0);
+  if (t >= total) return 0;
+  need_ready = false;
+  if (t >= sc->cum[cls][i + 1]) {          // past the op boundary: a later op of the class
+    while (t >= sc->cum[cls][i + 1]) ++i;
+    slot = sc->cls_slot[cls][i];
+    op = &a->ops[slot];
+    need_ready = true;
   }
+  const unsigned local = t - sc->cum[cls][i];
+  const unsigned d = t - h;
+  const bool hit = !need_ready && d < 32u;
+  int4 got;
+  got.x = __shfl_sync(0xffffffffu, e.x, hit ? d : 0);
+  got.y = __shfl_sync(0xffffffffu, e.y, hit ? d : 0);
+  got.z = __shfl_sync(0xffffffffu, e.z, hit ? d : 0);
+  got.w = __shfl_sync(0xffffffffu, e.w, hit ? d : 0);
+  if (!hit) got = op->tile_list[local];
+  ti.kind = entry_kind(got);
+  ti.n = entry_n(got);
+  ti.m = entry_m(got);
+  ti.row0 = got.y;
+  ti.rows = got.z;
+  ti.expert = got.w;
+  ti.slot = slot;
+  ti.tile = (int)local;
+  ti.cls = cls;
+  ti.kblocks = ti.kind == kCombine ? 0 : (ti.kind == kGateUp ? a->H : a->I) / kBlockK;
+  return 1;
 }
 
-// The decision at a tile boundary.  Returns with ti.kind == kEnd when nothing is left (or
-// the run was aborted).
-__device__ inline void claim_next(const Ctx& c, SharedCtl* sc, RunHead* rh, TileInfo& ti) {
+// The decision at a tile boundary (whole producer warp).  Returns with ti.kind == kEnd when
+// nothing is left (or the run was aborted).
+__device__ inline void claim_next(const Ctx& c, SharedCtl* sc, RunHead* rh, int lane, TileInfo& ti) {
   const RunArgs* a = c.a;
   unsigned long long t0 = 0;
   for (unsigned it = 0;; ++it) {
     if (aborted(c)) break;
     const int q = ld_volatile(&a->g->budget);
     const int first = ((int)blockIdx.x < q) ? MOE_CLASS_DECODE : MOE_CLASS_PREFILL;
-    const int r1 = try_claim(a, sc, rh, first, ti);
-    if (r1 == 1) { ti.t_claim = gtime_ns(); return; }
-    const int r2 = try_claim(a, sc, rh, 1 - first, ti);
-    if (r2 == 1) { ti.t_claim = gtime_ns(); return; }
+    bool need_ready = false;
+    int r1 = try_claim(a, sc, rh, first, lane, ti, need_ready);
+    int r2 = 0;
+    if (r1 != 1) r2 = try_claim(a, sc, rh, 1 - first, lane, ti, need_ready);
+    if (r1 == 1 || r2 == 1) {
+      ti.t_claim = gtime_ns();
+      if (need_ready) {                       // rare: wait (bounded) for the op to become ready
+        unsigned long long w0 = gtime_ns();
+        while (!op_ready(a, &a->ops[ti.slot])) {
+          __nanosleep(256);
+          if (aborted(c)) { ti.kind = kEnd; return; }
+          if ((long long)(gtime_ns() - w0) > a->wait_ns) {
+            if (lane == 0) report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, ti.slot, ti.tile);
+            ti.kind = kEnd;
+            return;
+          }
+        }
+      }
+      return;
+    }
     if (r1 == 0 && r2 == 0) break;
     __nanosleep(256);                         // an op exists but is not ready yet
     if ((it & 15u) == 15u) {
       const unsigned long long now = gtime_ns();
       if (t0 == 0) t0 = now;
       else if ((long long)(now - t0) > a->wait_ns) {
-        report(c.st, MOE_ETIMEOUT, 1, (int)blockIdx.x, r1, r2);
+        if (lane == 0) report(c.st, MOE_ETIMEOUT, 1, (int)blockIdx.x, r1, r2);
         break;
       }
     }
@@ -243,9 +278,14 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
   Ctx c{&args, &args.g->status};
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) { mbar_init(&sc->full[s], 1); mbar_init(&sc->empty[s], 1); }
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&sc->full[s], 1);
+      mbar_init(&sc->fullA[s], kGatherThreads);
+      mbar_init(&sc->empty[s], 1);
+    }
     for (int s = 0; s < 2; ++s) { mbar_init(&sc->tfull[s], 1); mbar_init(&sc->tempty[s], 128); }
-    for (int s = 0; s < kRing; ++s) { mbar_init(&sc->ifull[s], 1); mbar_init(&sc->iempty[s], 2); }
+    // a ring slot is released by the MMA warp, the epilogue and each of the gather warps
+    for (int s = 0; s < kRing; ++s) { mbar_init(&sc->ifull[s], 1); mbar_init(&sc->iempty[s], 2 + kGatherThreads / 32); }
     build_queues(&args, sc);
     sc->epi_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -264,22 +304,17 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
   const unsigned tmem = sc->tmem_base;
 
   if (warp == 0) {
-    // ============================================================ scheduler + producer
+    // ============================================================ scheduler + TMA producer
     int stage = 0, islot = 0;
     unsigned ph = 0, iph = 0;
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->iempty[islot], iph ^ 1u, 2))) break;
       TileInfo ti;
       ti.kind = kEnd;
-      if (lane == 0) claim_next(c, sc, rh, ti);
-      ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);
-      ti.slot = __shfl_sync(0xffffffffu, ti.slot, 0);
-      ti.m = __shfl_sync(0xffffffffu, ti.m, 0);
-      ti.n = __shfl_sync(0xffffffffu, ti.n, 0);
-      ti.row0 = __shfl_sync(0xffffffffu, ti.row0, 0);
-      ti.rows = __shfl_sync(0xffffffffu, ti.rows, 0);
-      ti.kblocks = __shfl_sync(0xffffffffu, ti.kblocks, 0);
-      ti.expert = __shfl_sync(0xffffffffu, ti.expert, 0);
+      ti.slot = ti.tile = ti.m = ti.row0 = ti.rows = ti.n = ti.kblocks = ti.expert = ti.cls = 0;
+      ti.t_claim = 0;
+      claim_next(c, sc, rh, lane, ti);
+      ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);      // the loops above exit warp-uniformly
       const OpDev* op = &args.ops[ti.kind == kEnd ? args.slots[0] : ti.slot];
       int ok = 1;
       if (lane == 0) {
@@ -297,36 +332,28 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
       if (ti.kind == kCombine) continue;
 
-      // rows this lane gathers (4 per gather4); rows past the tile's end repeat its last row
+      // Weight tiles by tiled TMA.  The A operand of a down tile is the packed intermediate:
+      // consecutive rows, one TMA box (8, 32 or 128 rows high, the smallest that holds the
+      // tile's rows); the A operand of a gate/up tile is gathered by the gather warps.
       const bool g1 = ti.kind == kGateUp;
-      const int n_g = (ti.rows + 3) >> 2;
-      int4 idx;
-      {
-        int r[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int p = ti.row0 + min(4 * lane + i, ti.rows - 1);
-          r[i] = g1 ? op->sorted_to_flat[p] / args.k : p;
-        }
-        idx = make_int4(r[0], r[1], r[2], r[3]);
-      }
-      const CUtensorMap* tma = g1 ? &op->tm_x : &op->tm_a;
       const CUtensorMap* tmw = g1 ? &op->tm_w1 : &op->tm_w2;
       const int wrow0 = g1 ? ti.expert * 2 * args.I + ti.n * kTileN1 : ti.expert * args.H + ti.n * kTileN2;
       const int wrow1 = g1 ? wrow0 + args.I : wrow0 + 128;
-      const unsigned tx = (unsigned)kBBytes + (unsigned)n_g * 512u;
+      const CUtensorMap* tma = ti.rows <= 8 ? &op->tm_a8 : (ti.rows <= 32 ? &op->tm_a32 : &op->tm_a128);
+      const unsigned abytes = g1 ? 0u : (ti.rows <= 8 ? 8u : (ti.rows <= 32 ? 32u : 128u)) * 128u;
+      const unsigned tx = (unsigned)kBBytes + abytes;
       bool fail = false;
       for (int kb = 0; kb < ti.kblocks; ++kb) {
         if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 5))) { fail = true; break; }
-        unsigned char* sA = stages + (size_t)stage * kStageBytes;
-        unsigned char* sB = sA + kABytes;
         if (lane == 0) {
+          unsigned char* sA = stages + (size_t)stage * kStageBytes;
+          unsigned char* sB = sA + kABytes;
           mbar_expect_tx(&sc->full[stage], tx);
           tma_tile_2d(sB, tmw, kb * kBlockK, wrow0, &sc->full[stage]);
           tma_tile_2d(sB + kBHalfBytes, tmw, kb * kBlockK, wrow1, &sc->full[stage]);
+          if (!g1) tma_tile_2d(sA, tma, kb * kBlockK, ti.row0, &sc->full[stage]);
         }
         __syncwarp();
-        if (lane < n_g) tma_gather4(sA + lane * 512, tma, kb * kBlockK, idx, &sc->full[stage]);
         if (++stage == kStages) { stage = 0; ph ^= 1u; }
       }
       if (fail) break;
@@ -334,7 +361,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
   } else if (warp == 1) {
     // ============================================================ MMA issuer
     int stage = 0, islot = 0, acc = 0;
-    unsigned ph = 0, iph = 0, aph[2] = {0, 0};
+    unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0;
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 6))) break;
       const int kind = sc->info[islot].kind;
@@ -347,8 +374,13 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         const unsigned d_tmem = tmem + (unsigned)acc * kAccCols;
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
+          if (kind == kGateUp) {       // gathered rows arrive through their own barrier
+            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], (phA >> stage) & 1u, 12))) { fail = true; break; }
+            phA ^= 1u << stage;
+          }
           tc_fence_after();
           if (lane == 0) {
+            fence_async_proxy_smem();                    // cp.async-written rows -> tensor core reads
             const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
             const unsigned long long ad = umma_desc(sA), bd = umma_desc(sA + kABytes);
 #pragma unroll
@@ -368,10 +400,67 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (lane == 0) mbar_arrive(&sc->iempty[islot]);
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
     }
+  } else if (warp < 2 + kGatherThreads / 32) {
+    // ============================================================ gather warps (cp.async)
+    // Rows of a gate/up tile are scattered tokens: row r of the tile is token
+    // sorted_to_flat[row0 + r] / k.  Eight lanes copy one 128-byte row slice (16 bytes each)
+    // into the 128-byte-swizzled layout the tensor core reads; each thread serves 8 rows.
+    const int gt = threadIdx.x - 64;
+    const int chunk = gt & 7, rbase = gt >> 3;            // rows rbase + 16 j, j = 0..7
+    int islot = 0;
+    unsigned iph = 0, kiter = 0;                          // kiter: k-blocks of all GEMM tiles so far
+    while (true) {
+      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 13))) break;
+      const int kind = sc->info[islot].kind;
+      const int kblocks = sc->info[islot].kblocks;
+      const int rows = sc->info[islot].rows, row0 = sc->info[islot].row0, slot = sc->info[islot].slot;
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sc->iempty[islot]);
+      if (++islot == kRing) { islot = 0; iph ^= 1u; }
+      if (kind == kEnd) break;
+      if (kind == kCombine) continue;
+      if (kind == kDown) {
+        // nothing to gather, but keep in step with the stage ring: a parity wait is only
+        // meaningful for a waiter that is at most one phase ahead of the barrier
+        bool failed = false;
+        for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
+          const int stage = (int)(kiter % kStages);
+          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kStages) & 1u) ^ 1u, 15))) { failed = true; break; }
+        }
+        if (failed) break;
+        continue;
+      }
+      const OpDev* op = &args.ops[slot];
+      const unsigned char* X = static_cast<const unsigned char*>(op->x);
+      const size_t pitch = (size_t)args.H * 2;
+      const unsigned char* src[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) {
+        const int r = rbase + 16 * j;
+        src[j] = nullptr;
+        if (r < rows) src[j] = X + (size_t)(op->sorted_to_flat[row0 + r] / args.k) * pitch + chunk * 16;
+      }
+      bool fail = false;
+      for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
+        const int stage = (int)(kiter % kStages);
+        const unsigned ph = (kiter / kStages) & 1u;
+        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 14))) { fail = true; break; }
+        const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          const int r = rbase + 16 * j;
+          if (src[j] != nullptr)
+            cp_async_16(sA + r * 128 + ((chunk ^ (r & 7)) << 4), src[j] + (size_t)kb * (kBlockK * 2));
+        }
+        cp_async_arrive_noinc(&sc->fullA[stage]);
+      }
+      if (fail) break;
+    }
+    cp_async_wait_all();
   } else {
-    // ============================================================ epilogue (warps 2..5)
+    // ============================================================ epilogue (warps 6..9)
     const int q = warp & 3;                       // TMEM lane quadrant this warp may read
-    const int etid = threadIdx.x - 64;            // 0..127
+    const int etid = threadIdx.x - (64 + kGatherThreads);   // 0..127
     int islot = 0, acc = 0;
     unsigned iph = 0, aph[2] = {0, 0};
     while (true) {

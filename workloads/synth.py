@@ -90,6 +90,13 @@ SPECS = {
     "c5": Spec("c5", Shape(256, 8, 6144, 2048, "fp8"), ((PREFILL, 4096), (DECODE, 512)),
                "zipf", 1.0, 1.0, 1.0, 5),
 }
+# profiling-size variants (same H, I, k and routing law; 64 experts, so that the weights are
+# 1.8 GB -- well above L2, small enough for a profiler to save and restore)
+SPECS["c2s"] = scaled_ = dataclasses.replace(SPECS["c2"], name="c2s", shape=Shape(64, 8, 3072, 1536),
+                                             ops=((DECODE, 32),))
+SPECS["c3s"] = dataclasses.replace(SPECS["c3"], name="c3s", shape=Shape(64, 8, 3072, 1536),
+                                   ops=((PREFILL, 2048),))
+del scaled_
 C4_BUDGETS = (16, 32, 64)     # decode SM budget cycled between layers
 
 
