@@ -153,6 +153,29 @@ int moe_read_tile_table(moe_ctx_t* ctx, int slot, int32_t* host_out, int max_til
  * returns how many were written in *n.  Synchronous. */
 int moe_read_tile_log(moe_ctx_t* ctx, moe_tile_rec_t* host_out, int max_records, int* n);
 
+/* The plan step for callers that must not allocate (no counterpart in the paper: it is a
+ * deployment convenience of this library).  Same counts / offsets / sorted_to_flat /
+ * flat_to_sorted as moe_plan, bit for bit, but without a context or a workspace: the
+ * histogram scratch is a fixed 128 KB device array inside the library image, held by every
+ * GPU that loads the library until the process exits.  It is meant for code that runs where
+ * a device allocation is not an option -- all memory belongs to another allocator, or the
+ * caller may not make calls that can synchronise the device, as cudaMalloc and cudaFree
+ * can.  The call itself allocates nothing and calls no allocating routine.
+ *   - limits: n_tokens * top_k <= MOE_PLAN_STATIC_MAX_ROWS and n_experts <=
+ *     MOE_PLAN_STATIC_MAX_EXPERTS, else MOE_ENOSPC (nothing is launched);
+ *   - all pointers are device pointers owned by the caller, sizes as in moe_op_t;
+ *   - expert ids outside [0, n_experts) are skipped silently (moe_plan reports them);
+ *   - the first call on each device looks up the scratch array's device address; make
+ *     that first call outside any stream capture;
+ *   - every call uses the same array, which keeps the previous call's contents (nothing
+ *     in it needs clearing between calls); calls whose kernels could overlap on the GPU
+ *     -- other streams, other host threads -- race on it and must be serialised. */
+#define MOE_PLAN_STATIC_MAX_ROWS 32768
+#define MOE_PLAN_STATIC_MAX_EXPERTS 256
+int moe_plan_static(const int32_t* topk_ids, int32_t n_tokens, int32_t top_k, int32_t n_experts,
+                    int32_t* counts, int32_t* offsets, int32_t* sorted_to_flat,
+                    int32_t* flat_to_sorted, void* stream);
+
 /* Multiprocessor count of the context's device (the default persistent grid). */
 int moe_sm_count(moe_ctx_t* ctx);
 

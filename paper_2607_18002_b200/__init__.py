@@ -28,7 +28,9 @@ MOE_TILE_M = 128
 
 EXPORTS = ("moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_run",
            "moe_combine", "moe_set_budget", "moe_status", "moe_footprint",
-           "moe_read_tile_table", "moe_read_tile_log", "moe_sm_count", "moe_strerror")
+           "moe_read_tile_table", "moe_read_tile_log", "moe_sm_count", "moe_strerror",
+           "moe_plan_static")
+MOE_PLAN_STATIC_MAX_ROWS, MOE_PLAN_STATIC_MAX_EXPERTS = 32768, 256
 
 
 class MoeError(RuntimeError):
@@ -91,6 +93,7 @@ def lib() -> C.CDLL:
         L.moe_footprint.argtypes = [vp, C.c_int, C.POINTER(i32), C.POINTER(i32)]
         L.moe_read_tile_table.argtypes = [vp, C.c_int, vp, C.c_int]
         L.moe_read_tile_log.argtypes = [vp, vp, C.c_int, C.POINTER(C.c_int)]
+        L.moe_plan_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
         L.moe_sm_count.argtypes = [vp]
         L.moe_strerror.argtypes = [C.c_int]
         L.moe_strerror.restype = C.c_char_p
@@ -175,6 +178,17 @@ def moe_read_tile_log(ctx: int, max_records: int) -> np.ndarray:
     _check(lib().moe_read_tile_log(C.c_void_p(ctx), out.ctypes.data_as(C.c_void_p), max_records,
                                    C.byref(n)), "moe_read_tile_log")
     return out[:n.value]
+
+
+def moe_plan_static(topk_ids_ptr: int, n_tokens: int, top_k: int, n_experts: int, counts_ptr: int,
+                    offsets_ptr: int, sorted_to_flat_ptr: int, flat_to_sorted_ptr: int,
+                    stream: int) -> None:
+    """The allocation-free plan: device pointers in, nothing allocated; see the header for
+    the size limits and the rule that calls sharing the built-in scratch must not overlap."""
+    _check(lib().moe_plan_static(C.c_void_p(topk_ids_ptr), n_tokens, top_k, n_experts,
+                                 C.c_void_p(counts_ptr), C.c_void_p(offsets_ptr),
+                                 C.c_void_p(sorted_to_flat_ptr), C.c_void_p(flat_to_sorted_ptr),
+                                 C.c_void_p(stream)), "moe_plan_static")
 
 
 def moe_sm_count(ctx: int) -> int:
