@@ -219,43 +219,71 @@ def oracle_sample(w: Workload, seconds_target: float = 12.0):
                            f"seeded tokens of {w.name} ({last_dt:.2f} s)")
 
 
-def tile_stats(w: Workload):
-    """Per-tile service times (claim -> commit) of the last launch of one extra step, from the
-    kernel's tile log: the analogue of the paper's preemption-interval measurement."""
-    w.step()
-    w.ctx.check()
-    log = w.ctx.tile_log()
-    if len(log) == 0:
-        return None
-    if os.environ.get("MOE_BENCH_DUMP_LOG"):
-        np.save(os.environ["MOE_BENCH_DUMP_LOG"], log)
+def _log_summary(log):
+    """Service time (claim -> commit) per class and tile kind, CTA occupancy and idle gaps."""
     out = {"records": int(len(log))}
+    if len(log) == 0:
+        return out
     t0 = int(log["t_claim"].min())
     span = (int(log["t_commit"].max()) - t0) / 1e3
     out["kernel_span_us"] = span
     service = (log["t_commit"].astype(np.int64) - log["t_claim"].astype(np.int64)) / 1e3
     names = {0: "gate_up", 1: "down", 2: "combine"}
     for cls, cname in ((0, "decode"), (1, "prefill")):
+        mc = log["cls"] == cls
+        if not mc.any():
+            continue
+        gemm = mc & (log["kind"] < 2)
+        if gemm.any():
+            v = service[gemm]
+            out[f"{cname}_tile"] = {"n": int(gemm.sum()), "p50_us": float(np.percentile(v, 50)),
+                                    "p99_us": float(np.percentile(v, 99)), "max_us": float(v.max())}
+        out[f"{cname}_op_us"] = float((int(log["t_commit"][mc].max()) - int(log["t_claim"][mc].min())) / 1e3)
+        out[f"{cname}_first_claim_us"] = float((int(log["t_claim"][mc].min()) - t0) / 1e3)
         for kind, kname in names.items():
-            m = (log["cls"] == cls) & (log["kind"] == kind)
+            m = mc & (log["kind"] == kind)
             if m.any():
                 v = service[m]
                 out[f"{cname}_{kname}"] = {"n": int(m.sum()), "p50_us": float(np.percentile(v, 50)),
-                                           "p99_us": float(np.percentile(v, 99)),
-                                           "max_us": float(v.max()), "mean_us": float(v.mean())}
-    n_cta = int(log["cta"].max()) + 1
-    out["occupancy"] = float(service.sum() / (n_cta * span)) if span > 0 else None
-    # idle time between a CTA's consecutive tiles (commit -> next claim)
-    gaps = []
-    for c in range(n_cta):
+                                           "p99_us": float(np.percentile(v, 99)), "mean_us": float(v.mean())}
+    ctas = np.unique(log["cta"])
+    out["ctas_with_tiles"] = int(len(ctas))
+    # busy time per CTA = union of its (overlapping) tile intervals
+    busy = 0.0
+    for c in ctas:
         r = log[log["cta"] == c]
-        r = r[np.argsort(r["t_claim"])]
-        if len(r) > 1:
-            gaps.append((r["t_claim"][1:].astype(np.int64) - r["t_commit"][:-1].astype(np.int64)) / 1e3)
-    if gaps:
-        g = np.concatenate(gaps)
-        out["gap_us"] = {"p50": float(np.percentile(g, 50)), "p99": float(np.percentile(g, 99)),
-                         "mean": float(g.mean())}
+        order = np.argsort(r["t_claim"])
+        a, b = r["t_claim"][order].astype(np.int64), r["t_commit"][order].astype(np.int64)
+        end = np.maximum.accumulate(b)
+        start_new = np.concatenate([[True], a[1:] > end[:-1]])
+        seg_start = a[start_new]
+        seg_end = np.concatenate([end[:-1][start_new[1:]], end[-1:]])
+        busy += float((seg_end - seg_start).sum()) / 1e3
+    out["queue_occupancy"] = busy / (len(ctas) * span) if span > 0 else None
+    return out
+
+
+def tile_stats(w: Workload):
+    """Per-tile timing of one extra (untimed) step from the kernel's tile log: the analogue of
+    the paper's preemption-interval measurement; for a co-scheduled workload also the decode
+    tiles alone (same budget, no prefill op in the launch) for the co-run / isolated ratio."""
+    w.step()
+    w.ctx.check()
+    log = w.ctx.tile_log()
+    if os.environ.get("MOE_BENCH_DUMP_LOG"):
+        np.save(os.environ["MOE_BENCH_DUMP_LOG"], log)
+    out = {"corun": _log_summary(log)}
+    _, bound, _ = w.layers[-1]
+    dec = [s for s, b in enumerate(bound) if b.c.cls == 0]
+    if dec and len(dec) < len(bound):
+        w.ctx.run(dec, fuse_combine=True)
+        w.ctx.check()
+        iso = _log_summary(w.ctx.tile_log())
+        out["decode_isolated"] = iso
+        if "decode_tile" in iso and "decode_tile" in out["corun"]:
+            out["decode_tile_p99_ratio"] = out["corun"]["decode_tile"]["p99_us"] / iso["decode_tile"]["p99_us"]
+            out["decode_tile_p50_ratio"] = out["corun"]["decode_tile"]["p50_us"] / iso["decode_tile"]["p50_us"]
+            out["decode_op_ratio"] = out["corun"]["decode_op_us"] / iso["decode_op_us"]
     return out
 
 
