@@ -15,10 +15,12 @@ constexpr int kTileM = MOE_TILE_M;   // token rows per tile (M_t)
 constexpr int kTileN1 = 128;         // SwiGLU output columns per gate/up tile (256 weight rows)
 constexpr int kTileN2 = 256;         // output columns per down-GEMM tile
 constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle row of bf16)
-constexpr int kStages = 4;           // shared-memory pipeline depth
+constexpr int kRowBytes = kBlockK * 2;
+constexpr int kStages = 3;           // shared-memory pipeline depth (64 KB per stage)
 constexpr int kCombineTokens = 32;   // tokens per combine tile
 constexpr int kPlanChunk = 256;      // routed rows ranked by one warp in the plan kernels
-constexpr int kGroupMTiles = 16;     // m-tiles per dependency group of the tile list
+constexpr int kGroupWork = 16;       // work tiles per dependency group of the tile list
+constexpr int kWorkRowsBf16 = 256;   // rows of a work tile: two m-tiles share each weight tile
 constexpr int kMaxOps = 16;
 constexpr int kMaxExperts = 1024;
 
@@ -59,6 +61,7 @@ struct __align__(128) OpDev {
   CUtensorMap tm_w1;    // [E*2I, H]   box {64, 128} gate/up weights
   CUtensorMap tm_w2;    // [E*H, I]    box {64, 128} down weights
   CUtensorMap tm_a128;  // [Rmax, I]   box {64, 128}
+  CUtensorMap tm_a256;  // [Rmax, I]   box {64, 256}
   int cls, n_tokens, n_rows, after_op;
   const void* x;
   const float* x_scale;
@@ -83,7 +86,7 @@ struct __align__(128) OpDev {
   int* plan_hist;        // [n_chunks, E] per-warp histogram, then per-warp base rank
   PlanState* plan;
   RunState* run;
-  int* g1_done;          // [max_mtiles] committed gate/up tiles per m-tile
+  int* g1_done;          // [max_mtiles] committed gate/up tiles per work tile
 };
 
 struct Status {   // first error wins (atomicCAS on code)
@@ -115,6 +118,9 @@ struct RunArgs {
   int n_ops;
   int fuse_combine;
   int E, k, H, I;
+#ifdef MOE_TIMING_PROBE
+  long long* dbg;
+#endif
   long long wait_ns;
   int slots[kMaxOps];
 };

@@ -10,7 +10,7 @@
 
 namespace moe {
 cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, int E, int NT1,
-                        int NT2, cudaStream_t stream);
+                        int NT2, int work_rows, cudaStream_t stream);
 cudaError_t launch_combine(const OpDev* d_op, int T, int k, int H, cudaStream_t stream);
 cudaError_t prepare_run_kernel();
 cudaError_t launch_run(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream);
@@ -102,7 +102,8 @@ struct moe_ctx {
 
 namespace {
 
-// 2-D bf16 tensor map: `rows` x `cols` row-major, box = box_rows x 64 columns, 128-byte swizzle
+// 2-D bf16 tensor map: `rows` x `cols` row-major, box = box_rows x kBlockK columns, swizzle
+// as wide as a box row
 int make_map(moe_ctx* ctx, CUtensorMap* out, const void* base, size_t rows, size_t cols,
              int box_rows) {
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -111,7 +112,8 @@ int make_map(moe_ctx* ctx, CUtensorMap* out, const void* base, size_t rows, size
   cuuint32_t estr[2] = {1, 1};
   CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
                            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           kRowBytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS ? MOE_OK : MOE_ECUDA;
 }
@@ -227,6 +229,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
     rc = make_map(ctx, &h.tm_a8, h.A, (size_t)L.max_rows, (size_t)c.inter, 8);
     if (!rc) rc = make_map(ctx, &h.tm_a32, h.A, (size_t)L.max_rows, (size_t)c.inter, 32);
     if (!rc) rc = make_map(ctx, &h.tm_a128, h.A, (size_t)L.max_rows, (size_t)c.inter, 128);
+    if (!rc) rc = make_map(ctx, &h.tm_a256, h.A, (size_t)L.max_rows, (size_t)c.inter, 256);
     if (!rc) rc = make_map(ctx, &h.tm_w1, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 128);
     if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
     if (rc) return rc;
@@ -235,7 +238,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   if (cudaMemcpyAsync(ctx->op_dev(slot), &h, sizeof(h), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ECUDA;
   if (launch_plan(ctx->op_dev(slot), ctx->g(), slot, op->n_tokens, c.top_k, c.n_experts, L.NT1, L.NT2,
-                  st) != cudaSuccess)
+                  kWorkRowsBf16, st) != cudaSuccess)
     return MOE_ECUDA;
   ctx->ops[slot] = *op;
   ctx->planned[slot] = true;
@@ -269,6 +272,10 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
   a.fuse_combine = fuse_combine ? 1 : 0;
   a.E = c.n_experts; a.k = c.top_k; a.H = c.hidden; a.I = c.inter;
   a.wait_ns = (long long)c.wait_limit_us * 1000;
+#ifdef MOE_TIMING_PROBE
+  a.dbg = reinterpret_cast<long long*>(ctx->ws + ctx->L.log_off);   // the tile log area doubles as probe buffer
+  a.log_cap = 0;
+#endif
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
   if (launch_run(a, ctx->rh(), ctx->n_ctas, st) != cudaSuccess) return MOE_ECUDA;
@@ -327,6 +334,9 @@ int moe_read_tile_log(moe_ctx_t* ctx, moe_tile_rec_t* host_out, int max_records,
   RunHead rh;
   if (cudaMemcpy(&rh, ctx->rh(), sizeof(rh), cudaMemcpyDeviceToHost) != cudaSuccess) return MOE_ECUDA;
   int cnt = (int)rh.log_count;
+#ifdef MOE_TIMING_PROBE
+  cnt = ctx->cfg.tile_log_entries;
+#endif
   if (cnt > ctx->cfg.tile_log_entries) cnt = ctx->cfg.tile_log_entries;
   if (cnt > max_records) cnt = max_records;
   if (cnt > 0 && cudaMemcpy(host_out, ctx->ws + ctx->L.log_off, (size_t)cnt * sizeof(moe_tile_rec_t),

@@ -76,11 +76,11 @@ __device__ inline int block_excl_scan(int v, int* total, int* warp_sums) {
 // ---------------------------------------------------------------- K2: scans + tile table + tile list
 __global__ void __launch_bounds__(1024)
 plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int NT1, int NT2,
-                 int T) {
+                 int T, int work_rows) {
   __shared__ int warp_sums[33];
   __shared__ int s_cnt[kMaxExperts], s_m0[kMaxExperts], s_grp[kMaxExperts], s_moff[kMaxExperts];
-  __shared__ int g_first[kMaxExperts], g_cnt[kMaxExperts], g_base1[kMaxExperts], g_base2[kMaxExperts];
-  __shared__ int s_ngroups, s_ntiles;
+  __shared__ int g_cnt[kMaxExperts], g_base1[kMaxExperts], g_base2[kMaxExperts];
+  __shared__ int s_ntiles;
   const int e = threadIdx.x;
 
   // column scan over the per-warp histograms: base rank of every (warp chunk, expert)
@@ -109,7 +109,6 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   int x_moe;
   const int m0 = block_excl_scan(me, &x_moe, warp_sums);
   if (e < E) {
-    s_m0[e] = m0;
     for (int j = 0; j < me; ++j) {
       MTile t;
       t.expert = e;
@@ -121,21 +120,26 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   }
   __syncthreads();
 
-  // dependency groups: consecutive experts holding at least kGroupMTiles m-tiles.  The
-  // list is  G1(g0) G1(g1) G2(g0) G1(g2) G2(g1) ... G2(last): every down-GEMM tile comes
-  // after all gate/up tiles of its group and of one more group, so by the time it is
-  // claimed the tiles it depends on were claimed long before.
+  // Work tiles (the unit the queues hand out): up to `work_rows` consecutive rows of one
+  // expert, i.e. one or two adjacent m-tiles that share each weight tile they read.
+  // Dependency groups: consecutive experts holding at least kGroupWork work tiles.  The list
+  // is  G1(g0) G1(g1) G2(g0) G1(g2) G2(g1) ... G2(last): every down-GEMM tile comes after all
+  // gate/up tiles of its group and of one more group, so by the time it is claimed the tiles
+  // it depends on were claimed long before.
+  const int we = (e < E) ? (cnt + work_rows - 1) / work_rows : 0;
+  int n_work;
+  const int w0 = block_excl_scan(we, &n_work, warp_sums);
+  if (e < E) s_m0[e] = w0;
+  __syncthreads();
   if (threadIdx.x == 0) {
-    int ng = 0, acc = 0, first = 0;
+    int ng = 0, acc = 0;
     for (int x = 0; x < E; ++x) {
-      const int m = (s_cnt[x] + kTileM - 1) / kTileM;
+      const int m = (s_cnt[x] + work_rows - 1) / work_rows;
       s_grp[x] = ng;
       s_moff[x] = acc;
       acc += m;
-      if (acc >= kGroupMTiles || x == E - 1) {
-        if (acc > 0) { g_first[ng] = first; g_cnt[ng] = acc; ++ng; }
-        else { /* trailing empty experts join nothing */ }
-        first += acc;
+      if (acc >= kGroupWork || x == E - 1) {
+        if (acc > 0) { g_cnt[ng] = acc; ++ng; }
         acc = 0;
       }
     }
@@ -146,20 +150,19 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
       if (gi >= 1) { g_base2[gi - 1] = pos; pos += g_cnt[gi - 1] * NT2; }
     }
     if (ng > 0) { g_base2[ng - 1] = pos; pos += g_cnt[ng - 1] * NT2; }
-    s_ngroups = ng;
     s_ntiles = pos;
   }
   __syncthreads();
 
-  for (int m = threadIdx.x; m < x_moe; m += blockDim.x) {
-    const MTile mt = op->mtiles[m];
-    const int ex = mt.expert;
-    const int gi = s_grp[ex];
-    const int Me = (s_cnt[ex] + kTileM - 1) / kTileM;
-    const int j = m - s_m0[ex];
-    const int b1 = g_base1[gi] + s_moff[ex] * NT1, b2 = g_base2[gi] + s_moff[ex] * NT2;
-    for (int n = 0; n < NT1; ++n) op->tile_list[b1 + n * Me + j] = make_entry(kGateUp, n, m, mt.row0, mt.rows, ex);
-    for (int n = 0; n < NT2; ++n) op->tile_list[b2 + n * Me + j] = make_entry(kDown, n, m, mt.row0, mt.rows, ex);
+  if (e < E && we > 0) {           // inside an expert: n-major over its work tiles
+    const int gi = s_grp[e];
+    const int b1 = g_base1[gi] + s_moff[e] * NT1, b2 = g_base2[gi] + s_moff[e] * NT2;
+    for (int j = 0; j < we; ++j) {
+      const int row0 = off + j * work_rows, rows = min(work_rows, cnt - j * work_rows);
+      const int m = w0 + j;
+      for (int n = 0; n < NT1; ++n) op->tile_list[b1 + n * we + j] = make_entry(kGateUp, n, m, row0, rows, e);
+      for (int n = 0; n < NT2; ++n) op->tile_list[b2 + n * we + j] = make_entry(kDown, n, m, row0, rows, e);
+    }
   }
   const int n_gemm = s_ntiles;
   const int n_comb = (T + kCombineTokens - 1) / kCombineTokens;
@@ -212,13 +215,13 @@ plan_scatter_kernel(const OpDev* __restrict__ op, int R, int E) {
 }
 
 cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, int E, int NT1,
-                        int NT2, cudaStream_t stream) {
+                        int NT2, int work_rows, cudaStream_t stream) {
   const int R = T * k;
   const int n_chunks = (R + kPlanChunk - 1) / kPlanChunk;
   const int blocks = (n_chunks + kPlanWarps - 1) / kPlanWarps;
   const size_t smem = (size_t)kPlanWarps * E * sizeof(int);
   if (blocks > 0) plan_hist_kernel<<<blocks, kPlanThreads, smem, stream>>>(d_op, g, slot, R, E);
-  plan_scan_kernel<<<1, 1024, 0, stream>>>(d_op, n_chunks, R, E, NT1, NT2, T);
+  plan_scan_kernel<<<1, 1024, 0, stream>>>(d_op, n_chunks, R, E, NT1, NT2, T, work_rows);
   if (blocks > 0) plan_scatter_kernel<<<blocks, kPlanThreads, smem, stream>>>(d_op, R, E);
   return cudaGetLastError();
 }

@@ -40,6 +40,12 @@ __device__ __forceinline__ void tma_tile_2d(void* dst, const CUtensorMap* tm, in
       "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
+// L2 prefetch of one tensor-map box: no shared memory, no barrier
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* tm, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(tm), "r"(x),
+               "r"(y)
+               : "memory");
+}
 __device__ __forceinline__ void tma_gather4(void* dst, const CUtensorMap* tm, int x, int4 rows,
                                             void* bar) {
   asm volatile(
@@ -118,14 +124,14 @@ __device__ __forceinline__ int ld_volatile(const int* p) {
   return *reinterpret_cast<const volatile int*>(p);
 }
 
-// UMMA shared-memory descriptor: K-major operand, 128-byte swizzle, rows of 128 bytes,
-// 8-row groups 1024 bytes apart.
-__device__ __forceinline__ unsigned long long umma_desc(unsigned saddr) {
+// UMMA shared-memory descriptor of a K-major operand whose rows are row_bytes (64 or 128)
+// wide and swizzled with the matching pattern; 8-row groups lie 8 * row_bytes apart.
+__device__ __forceinline__ unsigned long long umma_desc(unsigned saddr, unsigned row_bytes) {
   unsigned long long d = (unsigned long long)((saddr & 0x3ffffu) >> 4);
-  d |= 1ull << 16;                 // leading byte offset (unused for swizzled K-major)
-  d |= (1024ull >> 4) << 32;       // stride byte offset between 8-row groups
-  d |= 1ull << 46;                 // descriptor version (sm_100)
-  d |= 2ull << 61;                 // SWIZZLE_128B
+  d |= 1ull << 16;                                   // leading byte offset (unused for swizzled K-major)
+  d |= (unsigned long long)((8u * row_bytes) >> 4) << 32;   // stride byte offset between 8-row groups
+  d |= 1ull << 46;                                   // descriptor version (sm_100)
+  d |= (row_bytes == 128u ? 2ull : 4ull) << 61;      // SWIZZLE_128B : SWIZZLE_64B
   return d;
 }
 // instruction descriptor: D fp32, A/B bf16, both K-major, M = 128, N = 256

@@ -1,24 +1,27 @@
 // moe_run: the persistent expert kernel (the adaptive persistent kernel of Section 4 of the
 // paper, rebuilt for sm_100a).
 //
-// One CTA per SM, 10 warps with fixed roles:
-//   warp 0     scheduler + producer.  At every tile boundary it reads the decode budget
-//              word and the two queue heads, claims the next tile (decode first for CTAs
-//              below the budget, prefill first for the others, each falling back to the
-//              other class: Sections 4.2 and 5.4), hands the tile to the other warps
-//              through a shared-memory ring guarded by mbarriers (the hand-off of
-//              Section 4.3: the first pipeline warp decides, later warps follow), waits for
-//              the tile's dependencies, then feeds the pipeline: weight tiles (and the
-//              packed intermediate rows of a down tile) by tiled TMA.
-//   warp 1     issues tcgen05.mma (128 x 256 x 16, bf16 -> fp32) into one of two TMEM
-//              accumulators; tcgen05.commit releases pipeline stages and publishes the
-//              accumulator.
-//   warps 2-5  gather: the activation rows of a gate/up tile are scattered tokens; they are
-//              copied through the permutation with 16-byte cp.async into the swizzled
-//              layout the tensor core reads.
-//   warps 6-9  epilogue: tcgen05.ld, SwiGLU (gate/up tiles), bf16 stores, then the release
-//              of dependency counters, the op's done word and the tile log.  They also run
-//              the combine tiles.
+// One CTA per SM, 16 warps with fixed roles:
+//   warp 0      scheduler + producer.  At every tile boundary it reads the decode budget
+//               word and the two queue heads, claims the next tile (decode first for CTAs
+//               below the budget, prefill first for the others, each falling back to the
+//               other class: Sections 4.2 and 5.4), hands the tile to the other warps
+//               through a shared-memory ring guarded by mbarriers (the hand-off of
+//               Section 4.3: the first pipeline warp decides, later warps follow), waits for
+//               the tile's dependencies, then feeds the pipeline: weight tiles (and the
+//               packed intermediate rows of a down tile) by tiled TMA.
+//   warp 1      issues tcgen05.mma (128 x 256 x 16, bf16 -> fp32) into the TMEM accumulators;
+//               tcgen05.commit releases pipeline stages and publishes the accumulators.  A
+//               tile of up to 256 rows runs as two 128-row MMAs per k-step against the SAME
+//               weight tile in shared memory, which halves the weight bytes moved per flop.
+//   warp 2      committer: when the epilogue threads have stored a tile it fences and bumps the
+//               dependency counters, the op's done word and the tile log.
+//   warp 3      idle (it only joins the final barrier).
+//   warps 4-7   gather: the activation rows of a gate/up tile are scattered tokens; they are
+//               copied through the permutation with 16-byte cp.async into the swizzled
+//               layout the tensor core reads.
+//   warps 8-15  epilogue: tcgen05.ld, SwiGLU (gate/up tiles), bf16 stores transposed through
+//               shared memory into row segments.  They also run the combine tiles.
 // A phase switch happens only between tiles, so no accumulator, TMA transaction or buffer is
 // live across it (Section 4.2) and results are independent of the schedule.
 //
@@ -30,10 +33,11 @@
 namespace moe {
 
 constexpr int kGatherThreads = 128;                     // 4 gather warps
-constexpr int kThreads = 64 + kGatherThreads + 128;     // scheduler/TMA, MMA, gather x4, epilogue x4
-constexpr int kABytes = kTileM * kBlockK * 2;          // 16 KB activations per stage
-constexpr int kBHalfBytes = 128 * kBlockK * 2;         // 16 KB per 128 weight rows
-constexpr int kBBytes = 2 * kBHalfBytes;               // 32 KB weights per stage
+constexpr int kThreads = 512;                           // 16 warps, see the role list above
+constexpr int kAHalfBytes = kTileM * kRowBytes;        // 128 activation rows of one k-block
+constexpr int kABytes = 2 * kAHalfBytes;               // up to 256 activation rows per stage
+constexpr int kBHalfBytes = 128 * kRowBytes;           // 128 weight rows of one k-block
+constexpr int kBBytes = 2 * kBHalfBytes;               // 256 weight rows per stage
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kRing = 4;                               // tile-info ring depth
 constexpr int kAccCols = 256;                          // TMEM columns per accumulator
@@ -47,10 +51,10 @@ struct TileInfo {
 struct SharedCtl {
   unsigned long long full[kStages], fullA[kStages], empty[kStages];
   unsigned long long tfull[2], tempty[2];
-  unsigned long long ifull[kRing], iempty[kRing];
+  unsigned long long ifull[kRing], iempty[kRing], done[kRing];
   TileInfo info[kRing];
   unsigned tmem_base;
-  int epi_fail;
+  alignas(16) unsigned char epi_scratch[8][2048];   // per epilogue warp: 32 rows x 64 bytes
   int n_cls[2];
   int cls_slot[2][kMaxOps];
   unsigned cum[2][kMaxOps + 1];
@@ -263,11 +267,27 @@ __device__ inline void build_queues(const RunArgs* a, SharedCtl* sc) {
   }
 }
 
+// silu(g) * u through the hardware tanh approximation (one special-function op per element;
+// its error, |g| * 2.4e-4 at worst, stays below the bf16 rounding of the result)
 __device__ __forceinline__ float silu_mul(float g, float u) {
-  return g / (1.0f + __expf(-g)) * u;
+  float t;
+  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * g));
+  const float hg = 0.5f * g;
+  return fmaf(hg, t, hg) * u;                     // g * sigmoid(g) = g/2 * (1 + tanh(g/2))
 }
 
 // ------------------------------------------------------------------ the persistent kernel
+// which accumulator(s) a tile uses: a tile of up to 128 rows alternates between the two, a
+// tile of up to 256 rows takes both (rows 0..127 -> accumulator 0, rows 128..255 -> 1).
+// Every role walks the same tile sequence, so each derives this locally.
+struct AccUse {
+  int next = 0;
+  __device__ __forceinline__ void take(int rows, bool& use0, bool& use1) {
+    if (rows > kTileM) { use0 = use1 = true; }
+    else { use0 = next == 0; use1 = !use0; next ^= 1; }
+  }
+};
+
 __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_constant__ RunArgs args,
                                                               RunHead* rh) {
   extern __shared__ unsigned char smem_raw[];
@@ -283,11 +303,14 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       mbar_init(&sc->fullA[s], kGatherThreads);
       mbar_init(&sc->empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) { mbar_init(&sc->tfull[s], 1); mbar_init(&sc->tempty[s], 128); }
-    // a ring slot is released by the MMA warp, the epilogue and each of the gather warps
-    for (int s = 0; s < kRing; ++s) { mbar_init(&sc->ifull[s], 1); mbar_init(&sc->iempty[s], 2 + kGatherThreads / 32); }
+    for (int s = 0; s < 2; ++s) { mbar_init(&sc->tfull[s], 1); mbar_init(&sc->tempty[s], 256); }
+    // a ring slot is released by the MMA warp, the committer and each gather warp
+    for (int s = 0; s < kRing; ++s) {
+      mbar_init(&sc->ifull[s], 1);
+      mbar_init(&sc->iempty[s], 2 + kGatherThreads / 32);
+      mbar_init(&sc->done[s], 256);
+    }
     build_queues(&args, sc);
-    sc->epi_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_proxy();
   }
@@ -305,6 +328,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 
   if (warp == 0) {
     // ============================================================ scheduler + TMA producer
+#ifdef MOE_TIMING_PROBE
+    int dbg_i = 0;
+#endif
     int stage = 0, islot = 0;
     unsigned ph = 0, iph = 0;
     while (true) {
@@ -333,19 +359,22 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (ti.kind == kCombine) continue;
 
       // Weight tiles by tiled TMA.  The A operand of a down tile is the packed intermediate:
-      // consecutive rows, one TMA box (8, 32 or 128 rows high, the smallest that holds the
+      // consecutive rows, one TMA box (8, 32, 128 or 256 rows high, the smallest that holds the
       // tile's rows); the A operand of a gate/up tile is gathered by the gather warps.
       const bool g1 = ti.kind == kGateUp;
       const CUtensorMap* tmw = g1 ? &op->tm_w1 : &op->tm_w2;
       const int wrow0 = g1 ? ti.expert * 2 * args.I + ti.n * kTileN1 : ti.expert * args.H + ti.n * kTileN2;
       const int wrow1 = g1 ? wrow0 + args.I : wrow0 + 128;
-      const CUtensorMap* tma = ti.rows <= 8 ? &op->tm_a8 : (ti.rows <= 32 ? &op->tm_a32 : &op->tm_a128);
-      const unsigned abytes = g1 ? 0u : (ti.rows <= 8 ? 8u : (ti.rows <= 32 ? 32u : 128u)) * 128u;
-      const unsigned tx = (unsigned)kBBytes + abytes;
+      const int box = ti.rows <= 8 ? 8 : (ti.rows <= 32 ? 32 : (ti.rows <= 128 ? 128 : 256));
+      const CUtensorMap* tma = box == 8 ? &op->tm_a8 : (box == 32 ? &op->tm_a32 : (box == 128 ? &op->tm_a128 : &op->tm_a256));
+      const unsigned tx = (unsigned)kBBytes + (g1 ? 0u : (unsigned)(box * kRowBytes));
       bool fail = false;
       for (int kb = 0; kb < ti.kblocks; ++kb) {
         if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 5))) { fail = true; break; }
         if (lane == 0) {
+#ifdef MOE_TIMING_PROBE
+          if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 0] = clock64();
+#endif
           unsigned char* sA = stages + (size_t)stage * kStageBytes;
           unsigned char* sB = sA + kABytes;
           mbar_expect_tx(&sc->full[stage], tx);
@@ -360,18 +389,27 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     }
   } else if (warp == 1) {
     // ============================================================ MMA issuer
-    int stage = 0, islot = 0, acc = 0;
+#ifdef MOE_TIMING_PROBE
+    int dbg_i = 0;
+#endif
+    int stage = 0, islot = 0;
     unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0;
+    AccUse accs;
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 6))) break;
       const int kind = sc->info[islot].kind;
       const int kblocks = sc->info[islot].kblocks;
+      const int rows = sc->info[islot].rows;
       if (kind == kEnd) break;
       bool fail = false;
       if (kind != kCombine) {
-        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[acc], aph[acc] ^ 1u, 7))) break;
+        bool use0, use1;
+        accs.take(rows, use0, use1);
+        if (use0 && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[0], aph[0] ^ 1u, 7))) break;
+        if (use1 && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[1], aph[1] ^ 1u, 7))) break;
         tc_fence_after();
-        const unsigned d_tmem = tmem + (unsigned)acc * kAccCols;
+        const bool pair = use0 && use1;
+        const unsigned d0 = tmem + (use0 ? 0u : (unsigned)kAccCols);     // accumulator of rows 0..127
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
           if (kind == kGateUp) {       // gathered rows arrive through their own barrier
@@ -380,33 +418,51 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           }
           tc_fence_after();
           if (lane == 0) {
+#ifdef MOE_TIMING_PROBE
+            if (blockIdx.x == 7 && dbg_i < 4096) { args.dbg[dbg_i * 4 + 1] = clock64(); args.dbg[dbg_i * 4 + 2] = kind * 1000 + rows; }
+#endif
             fence_async_proxy_smem();                    // cp.async-written rows -> tensor core reads
             const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
-            const unsigned long long ad = umma_desc(sA), bd = umma_desc(sA + kABytes);
+            const unsigned long long ad = umma_desc(sA, kRowBytes), bd = umma_desc(sA + kABytes, kRowBytes);
 #pragma unroll
             for (int k4 = 0; k4 < kBlockK / 16; ++k4)   // +32 bytes along K per step (>>4 = 2)
-              tc_mma_bf16(d_tmem, ad + 2ull * k4, bd + 2ull * k4, kIdesc, (kb | k4) ? 1u : 0u);
+              tc_mma_bf16(d0, ad + 2ull * k4, bd + 2ull * k4, kIdesc, (kb | k4) ? 1u : 0u);
+            if (pair) {                                  // rows 128..255 against the same weight tile
+              const unsigned long long ad1 = umma_desc(sA + kAHalfBytes, kRowBytes);
+#pragma unroll
+              for (int k4 = 0; k4 < kBlockK / 16; ++k4)
+                tc_mma_bf16(tmem + (unsigned)kAccCols, ad1 + 2ull * k4, bd + 2ull * k4, kIdesc, (kb | k4) ? 1u : 0u);
+            }
             tc_commit(&sc->empty[stage]);               // frees the stage when the MMAs retire
+#ifdef MOE_TIMING_PROBE
+            if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 3] = clock64();
+#endif
           }
           __syncwarp();
           if (++stage == kStages) { stage = 0; ph ^= 1u; }
         }
         if (fail) break;
-        if (lane == 0) tc_commit(&sc->tfull[acc]);       // accumulator complete
+        if (lane == 0) {                                 // accumulator(s) complete
+          if (use0) tc_commit(&sc->tfull[0]);
+          if (use1) tc_commit(&sc->tfull[1]);
+        }
         __syncwarp();
-        aph[acc] ^= 1u;
-        acc ^= 1;
+        if (use0) aph[0] ^= 1u;
+        if (use1) aph[1] ^= 1u;
       }
       if (lane == 0) mbar_arrive(&sc->iempty[islot]);
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
     }
-  } else if (warp < 2 + kGatherThreads / 32) {
+  } else if (warp >= 4 && warp < 4 + kGatherThreads / 32) {
     // ============================================================ gather warps (cp.async)
     // Rows of a gate/up tile are scattered tokens: row r of the tile is token
-    // sorted_to_flat[row0 + r] / k.  Eight lanes copy one 128-byte row slice (16 bytes each)
-    // into the 128-byte-swizzled layout the tensor core reads; each thread serves 8 rows.
-    const int gt = threadIdx.x - 64;
-    const int chunk = gt & 7, rbase = gt >> 3;            // rows rbase + 16 j, j = 0..7
+    // sorted_to_flat[row0 + r] / k.  Adjacent lanes copy one row slice (16 bytes each)
+    // into the swizzled layout the tensor core reads.
+    const int gt = threadIdx.x - 128;
+    constexpr int kCpr = kRowBytes / 16;                  // 16-byte chunks per row slice
+    constexpr int kRowsPerPass = kGatherThreads / kCpr;   // rows covered by one cp.async per thread
+    constexpr int kPasses = 256 / kRowsPerPass;
+    const int chunk = gt % kCpr, rbase = gt / kCpr;       // rows rbase + kRowsPerPass * j
     int islot = 0;
     unsigned iph = 0, kiter = 0;                          // kiter: k-blocks of all GEMM tiles so far
     while (true) {
@@ -431,14 +487,13 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         continue;
       }
       const OpDev* op = &args.ops[slot];
-      const unsigned char* X = static_cast<const unsigned char*>(op->x);
+      const unsigned char* X = static_cast<const unsigned char*>(op->x) + chunk * 16;
       const size_t pitch = (size_t)args.H * 2;
-      const unsigned char* src[8];
+      int tok[kPasses];
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {
-        const int r = rbase + 16 * j;
-        src[j] = nullptr;
-        if (r < rows) src[j] = X + (size_t)(op->sorted_to_flat[row0 + r] / args.k) * pitch + chunk * 16;
+      for (int j = 0; j < kPasses; ++j) {
+        const int r = rbase + kRowsPerPass * j;
+        tok[j] = r < rows ? op->sorted_to_flat[row0 + r] / args.k : -1;
       }
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
@@ -446,99 +501,129 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         const unsigned ph = (kiter / kStages) & 1u;
         if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 14))) { fail = true; break; }
         const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
+        const unsigned char* Xk = X + (size_t)kb * (kBlockK * 2);
 #pragma unroll
-        for (int j = 0; j < 8; ++j) {
-          const int r = rbase + 16 * j;
-          if (src[j] != nullptr)
-            cp_async_16(sA + r * 128 + ((chunk ^ (r & 7)) << 4), src[j] + (size_t)kb * (kBlockK * 2));
+        for (int j = 0; j < kPasses; ++j) {
+          const int r = rbase + kRowsPerPass * j;
+          // the swizzle XORs the 16-byte chunk index with the row's position in its 8-row group
+          const int sw = kRowBytes == 128 ? (r & 7) : ((r >> 1) & 3);
+          if (tok[j] >= 0)
+            cp_async_16(sA + r * kRowBytes + ((chunk ^ sw) << 4), Xk + (size_t)tok[j] * pitch);
         }
         cp_async_arrive_noinc(&sc->fullA[stage]);
       }
       if (fail) break;
     }
     cp_async_wait_all();
-  } else {
-    // ============================================================ epilogue (warps 6..9)
-    const int q = warp & 3;                       // TMEM lane quadrant this warp may read
-    const int etid = threadIdx.x - (64 + kGatherThreads);   // 0..127
-    int islot = 0, acc = 0;
-    unsigned iph = 0, aph[2] = {0, 0};
+  } else if (warp == 2) {
+    // ============================================================ committer
+    // Publishes a tile once all epilogue threads have arrived on the tile's barrier: the
+    // barrier orders their stores before this warp's fence and release (cumulativity).
+    int islot = 0;
+    unsigned iph = 0;
     while (true) {
-      // A failed wait must not leave the other epilogue warps alone at the named barrier
-      // below: a warp that gives up records it in shared memory and still joins the barrier;
-      // all four warps leave together after it.
-      bool ok = __all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 9));
+      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 16))) break;
       TileInfo ti;
-      ti.kind = kEnd;
-      if (ok) ti = sc->info[islot];
-      OpDev* op = &args.ops[ti.kind == kEnd ? args.slots[0] : ti.slot];
+      if (lane == 0) ti = sc->info[islot];
+      const int kind = __shfl_sync(0xffffffffu, lane == 0 ? ti.kind : 0, 0);
+      if (kind == kEnd) break;
+      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->done[islot], iph, 17))) break;
+      if (lane == 0) {
+        commit_tile(c, rh, ti);
+        mbar_arrive(&sc->iempty[islot]);
+      }
+      __syncwarp();
+      if (++islot == kRing) { islot = 0; iph ^= 1u; }
+    }
+  } else if (warp >= 8) {
+    // ============================================================ epilogue (8 warps)
+    // Warp w may read TMEM lanes 32 (w % 4) .. +31, i.e. accumulator rows of that quadrant.
+    // The two warps of a quadrant split the columns of every accumulator the tile used.
+    const int q = warp & 3;
+    const int half = (warp - 8) >> 2;             // which half of the columns
+    const int etid = threadIdx.x - 256;           // 0..255
+    int islot = 0;
+    unsigned iph = 0, aph[2] = {0, 0};
+    AccUse accs;
+    unsigned char* scratch = sc->epi_scratch[warp - 8];
+    const int srow = lane >> 2, schunk = lane & 3;          // this lane's part of a store
+    while (true) {
+      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 9))) break;
+      const TileInfo ti = sc->info[islot];
+      if (ti.kind == kEnd) break;
+      OpDev* op = &args.ops[ti.slot];
+      bool ok = true;
       if (ti.kind == kCombine) {
-        combine_tokens(op, ti.row0, ti.row0 + ti.rows, args.k, args.H, etid, 128);
-      } else if (ti.kind != kEnd) {
-        ok = __all_sync(0xffffffffu, mbar_wait(c, &sc->tfull[acc], aph[acc], 10));
-        if (ok) {
+        combine_tokens(op, ti.row0, ti.row0 + ti.rows, args.k, args.H, etid, 256);
+      } else {
+        bool use[2];
+        accs.take(ti.rows, use[0], use[1]);
+        const bool pair = use[0] && use[1];
+        const bool g1 = ti.kind == kGateUp;
+        const int passes = (g1 ? kTileN1 : kTileN2) / 64;      // 32-column passes per warp
+        const size_t pitch = (size_t)(g1 ? args.I : args.H) * 2;
+#pragma unroll
+        for (int b = 0; b < 2; ++b) {
+          if (!use[b]) continue;
+          ok = __all_sync(0xffffffffu, mbar_wait(c, &sc->tfull[b], aph[b], 10));
+          if (!ok) break;
+          aph[b] ^= 1u;
           tc_fence_after();
-          const int row = q * 32 + lane;
-          const bool valid = row < ti.rows;
-          const unsigned taddr = tmem + (unsigned)acc * kAccCols + ((unsigned)(q * 32) << 16);
-          if (q * 32 < ti.rows) {
-            if (ti.kind == kGateUp) {
-              __nv_bfloat16* dst = op->A + (size_t)(ti.row0 + row) * args.I + ti.n * kTileN1;
+          const int rbase = pair ? b * kTileM : 0;               // first tile row of this accumulator
+          const int nrows = min(ti.rows - rbase, kTileM);
+          if (q * 32 < nrows) {
+            // 32 output columns (64 bytes of bf16) per pass.  Each lane owns one accumulator
+            // row; the warp transposes the pass through its shared-memory scratch so that a
+            // store instruction writes 8 rows x 64 contiguous bytes instead of 32 x 16.
+            const unsigned taddr = tmem + (unsigned)b * kAccCols + ((unsigned)(q * 32) << 16);
+            unsigned char* out = reinterpret_cast<unsigned char*>(g1 ? (void*)op->A : (void*)op->D) +
+                                 (size_t)(ti.row0 + rbase + q * 32) * pitch +
+                                 (size_t)ti.n * (g1 ? kTileN1 : kTileN2) * 2;
+            const int rows_here = min(32, nrows - q * 32);
 #pragma unroll 1
-              for (int cch = 0; cch < kTileN1 / 32; ++cch) {
+            for (int p = 0; p < passes; ++p) {
+              const int pass = half * passes + p;
+              uint4 o[4];
+              __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(o);
+              if (g1) {
                 unsigned g[32], u[32];
-                tc_ld32(taddr + cch * 32, g);
-                tc_ld32(taddr + 128 + cch * 32, u);
+                tc_ld32(taddr + pass * 32, g);
+                tc_ld32(taddr + 128 + pass * 32, u);
                 tc_wait_ld();
-                uint4 o[4];
-                __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(o);
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                   const float a0 = silu_mul(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i]));
                   const float a1 = silu_mul(__uint_as_float(g[2 * i + 1]), __uint_as_float(u[2 * i + 1]));
                   oh[i] = __floats2bfloat162_rn(a0, a1);
                 }
-                if (valid) {
-                  uint4* d4 = reinterpret_cast<uint4*>(dst + cch * 32);
-#pragma unroll
-                  for (int i = 0; i < 4; ++i) d4[i] = o[i];
-                }
-              }
-            } else {
-              __nv_bfloat16* dst = op->D + (size_t)(ti.row0 + row) * args.H + ti.n * kTileN2;
-#pragma unroll 1
-              for (int cch = 0; cch < kTileN2 / 32; ++cch) {
+              } else {
                 unsigned v[32];
-                tc_ld32(taddr + cch * 32, v);
+                tc_ld32(taddr + pass * 32, v);
                 tc_wait_ld();
-                uint4 o[4];
-                __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(o);
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
                   oh[i] = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-                if (valid) {
-                  uint4* d4 = reinterpret_cast<uint4*>(dst + cch * 32);
+              }
+              __syncwarp();                                          // scratch free again
 #pragma unroll
-                  for (int i = 0; i < 4; ++i) d4[i] = o[i];
-                }
+              for (int j = 0; j < 4; ++j)     // row `lane`, 16-byte chunk j (XOR keeps banks apart)
+                *reinterpret_cast<uint4*>(scratch + lane * 64 + ((j ^ ((lane >> 1) & 3)) << 4)) = o[j];
+              __syncwarp();
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int r = 8 * j + srow;
+                const uint4 v4 = *reinterpret_cast<const uint4*>(scratch + r * 64 + ((schunk ^ ((r >> 1) & 3)) << 4));
+                if (r < rows_here)
+                  *reinterpret_cast<uint4*>(out + (size_t)r * pitch + pass * 64 + schunk * 16) = v4;
               }
             }
           }
           tc_fence_before();
-          mbar_arrive(&sc->tempty[acc]);          // accumulator may be overwritten
-          aph[acc] ^= 1u;
-          acc ^= 1;
+          mbar_arrive(&sc->tempty[b]);            // accumulator may be overwritten
         }
       }
-      if (!ok) *reinterpret_cast<volatile int*>(&sc->epi_fail) = 1;
-      __threadfence();
-      fence_async_proxy();
-      asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (*reinterpret_cast<volatile int*>(&sc->epi_fail) != 0 || ti.kind == kEnd) break;
-      if (etid == 0) {
-        commit_tile(c, rh, ti);
-        mbar_arrive(&sc->iempty[islot]);
-      }
+      if (!ok) break;
+      mbar_arrive(&sc->done[islot]);              // this thread's part of the tile is stored
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
     }
   }
