@@ -42,6 +42,9 @@ constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kRing = 4;                               // tile-info ring depth
 constexpr int kAccCols = 256;                          // TMEM columns per accumulator
 constexpr int kEnd = -1;
+constexpr int kClaimAt = 2;                             // claim the next tile after this k-block
+constexpr int kAheadPrefetch = 3;                       // k-blocks of the next tile prefetched into L2
+constexpr int kPrefetchLead = 6;                        // ... this many k-blocks before the current tile ends
 
 struct TileInfo {
   int kind, slot, tile, m, row0, rows, n, kblocks, expert, cls;
@@ -57,6 +60,7 @@ struct SharedCtl {
   alignas(16) unsigned char epi_scratch[8][2048];   // per epilogue warp: 32 rows x 64 bytes
   int n_cls[2];
   int cls_slot[2][kMaxOps];
+  int cls_free[2][kMaxOps];        // 1: the op has no ready word and no predecessor
   unsigned cum[2][kMaxOps + 1];
 };
 
@@ -126,18 +130,18 @@ __device__ inline bool op_ready(const RunArgs* a, const OpDev* op) {
 // the price is that a ticket can land just past an op boundary, in an op that is not ready
 // yet -- the caller then waits for it (bounded), holding only tickets whose predecessors in
 // the queue are all claimed already.
-__device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, int cls, int lane,
-                                TileInfo& ti, bool& need_ready) {
+__device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, int cls, unsigned h,
+                                int lane, TileInfo& ti, bool& need_ready) {
   const int n = sc->n_cls[cls];
   if (n == 0) return 0;
   const unsigned total = sc->cum[cls][n];
-  const unsigned h = *reinterpret_cast<volatile unsigned*>(&rh->heads[cls]);
+  h = __shfl_sync(0xffffffffu, h, 0);       // one peek for the whole warp: lanes index entries by it
   if (h >= total) return 0;
   int i = 0;
   while (h >= sc->cum[cls][i + 1]) ++i;
   int slot = sc->cls_slot[cls][i];
   const OpDev* op = &a->ops[slot];
-  if (!op_ready(a, op)) return -1;
+  if (!sc->cls_free[cls][i] && !op_ready(a, op)) return -1;
   // the 32 entries from the head on are fetched while the fetch-add is in flight
   const unsigned base = h - sc->cum[cls][i];
   const unsigned n_op = sc->cum[cls][i + 1] - sc->cum[cls][i];
@@ -152,7 +156,7 @@ __device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, in
     while (t >= sc->cum[cls][i + 1]) ++i;
     slot = sc->cls_slot[cls][i];
     op = &a->ops[slot];
-    need_ready = true;
+    need_ready = !sc->cls_free[cls][i];
   }
   const unsigned local = t - sc->cum[cls][i];
   const unsigned d = t - h;
@@ -176,42 +180,60 @@ __device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, in
   return 1;
 }
 
-// The decision at a tile boundary (whole producer warp).  Returns with ti.kind == kEnd when
-// nothing is left (or the run was aborted).
-__device__ inline void claim_next(const Ctx& c, SharedCtl* sc, RunHead* rh, int lane, TileInfo& ti) {
+// One pass of the decision at a tile boundary (whole producer warp): 1 = claimed, 0 = both
+// queues exhausted, -1 = something exists but is not ready yet.  The abort word, the budget
+// word and both queue heads are loaded together (one round trip), then at most one
+// fetch-add per class.
+__device__ inline int claim_once(const Ctx& c, SharedCtl* sc, RunHead* rh, int lane, TileInfo& ti,
+                                 bool& need_ready) {
   const RunArgs* a = c.a;
+  const int ab = ld_volatile(&c.st->abort);
+  const int q = ld_volatile(&a->g->budget);
+  const unsigned h0 = *reinterpret_cast<volatile unsigned*>(&rh->heads[0]);
+  const unsigned h1 = *reinterpret_cast<volatile unsigned*>(&rh->heads[1]);
+  if (ab != 0) return 0;
+  const int first = ((int)blockIdx.x < q) ? MOE_CLASS_DECODE : MOE_CLASS_PREFILL;
+  need_ready = false;
+  const int r1 = try_claim(a, sc, rh, first, first == 0 ? h0 : h1, lane, ti, need_ready);
+  int r2 = 0;
+  if (r1 != 1) r2 = try_claim(a, sc, rh, 1 - first, first == 0 ? h1 : h0, lane, ti, need_ready);
+  if (r1 == 1 || r2 == 1) {
+    ti.t_claim = gtime_ns();
+    return 1;
+  }
+  return (r1 == 0 && r2 == 0) ? 0 : -1;
+}
+
+// A ticket that landed in an op that is not ready yet: wait for it (bounded).
+__device__ inline bool wait_op_ready(const Ctx& c, int lane, const TileInfo& ti) {
+  const RunArgs* a = c.a;
+  const unsigned long long w0 = gtime_ns();
+  while (!op_ready(a, &a->ops[ti.slot])) {
+    __nanosleep(256);
+    if (aborted(c)) return false;
+    if ((long long)(gtime_ns() - w0) > a->wait_ns) {
+      if (lane == 0) report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, ti.slot, ti.tile);
+      return false;
+    }
+  }
+  return true;
+}
+
+// Blocking form: waits (bounded) while an op exists that is not ready.  Returns with
+// ti.kind == kEnd when nothing is left (or the run was aborted).
+__device__ inline void claim_next(const Ctx& c, SharedCtl* sc, RunHead* rh, int lane, TileInfo& ti,
+                                  bool& need_ready) {
   unsigned long long t0 = 0;
   for (unsigned it = 0;; ++it) {
-    if (aborted(c)) break;
-    const int q = ld_volatile(&a->g->budget);
-    const int first = ((int)blockIdx.x < q) ? MOE_CLASS_DECODE : MOE_CLASS_PREFILL;
-    bool need_ready = false;
-    int r1 = try_claim(a, sc, rh, first, lane, ti, need_ready);
-    int r2 = 0;
-    if (r1 != 1) r2 = try_claim(a, sc, rh, 1 - first, lane, ti, need_ready);
-    if (r1 == 1 || r2 == 1) {
-      ti.t_claim = gtime_ns();
-      if (need_ready) {                       // rare: wait (bounded) for the op to become ready
-        unsigned long long w0 = gtime_ns();
-        while (!op_ready(a, &a->ops[ti.slot])) {
-          __nanosleep(256);
-          if (aborted(c)) { ti.kind = kEnd; return; }
-          if ((long long)(gtime_ns() - w0) > a->wait_ns) {
-            if (lane == 0) report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, ti.slot, ti.tile);
-            ti.kind = kEnd;
-            return;
-          }
-        }
-      }
-      return;
-    }
-    if (r1 == 0 && r2 == 0) break;
+    const int r = claim_once(c, sc, rh, lane, ti, need_ready);
+    if (r == 1) return;
+    if (r == 0) break;
     __nanosleep(256);                         // an op exists but is not ready yet
     if ((it & 15u) == 15u) {
       const unsigned long long now = gtime_ns();
       if (t0 == 0) t0 = now;
-      else if ((long long)(now - t0) > a->wait_ns) {
-        if (lane == 0) report(c.st, MOE_ETIMEOUT, 1, (int)blockIdx.x, r1, r2);
+      else if ((long long)(now - t0) > c.a->wait_ns) {
+        if (lane == 0) report(c.st, MOE_ETIMEOUT, 1, (int)blockIdx.x, 0, 0);
         break;
       }
     }
@@ -249,6 +271,9 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
       unsigned smid;
       asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
       r.sm = (int16_t)smid;
+#ifdef MOE_LOG_ROWS
+      r.sm = (int16_t)ti.rows;
+#endif
       a->log[idx] = r;
     }
   }
@@ -263,6 +288,7 @@ __device__ inline void build_queues(const RunArgs* a, SharedCtl* sc) {
     const int cls = op->cls;
     const int j = sc->n_cls[cls]++;
     sc->cls_slot[cls][j] = slot;
+    sc->cls_free[cls][j] = (op->ready == nullptr && op->after_op < 0) ? 1 : 0;
     sc->cum[cls][j + 1] = sc->cum[cls][j] + (unsigned)op_total_tiles(op, a->fuse_combine);
   }
 }
@@ -328,20 +354,27 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 
   if (warp == 0) {
     // ============================================================ scheduler + TMA producer
+    // The next tile is claimed while the current one is still being loaded (after its
+    // kClaimAt-th k-block), so the claim's round trips and the first loads of the next tile
+    // overlap the current tile's tail instead of draining the pipeline.  A CTA therefore
+    // holds at most one claimed tile beyond the one it is executing.
 #ifdef MOE_TIMING_PROBE
     int dbg_i = 0;
 #endif
     int stage = 0, islot = 0;
     unsigned ph = 0, iph = 0;
+    TileInfo ti, nx;
+    bool ti_need_ready = false, nx_need_ready = false, have_nx = false;
+    ti.kind = kEnd;
+    ti.slot = ti.tile = ti.m = ti.row0 = ti.rows = ti.n = ti.kblocks = ti.expert = ti.cls = 0;
+    ti.t_claim = 0;
+    nx = ti;
+    claim_next(c, sc, rh, lane, ti, ti_need_ready);
     while (true) {
+      ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);      // the claim loops exit warp-uniformly
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->iempty[islot], iph ^ 1u, 2))) break;
-      TileInfo ti;
-      ti.kind = kEnd;
-      ti.slot = ti.tile = ti.m = ti.row0 = ti.rows = ti.n = ti.kblocks = ti.expert = ti.cls = 0;
-      ti.t_claim = 0;
-      claim_next(c, sc, rh, lane, ti);
-      ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);      // the loops above exit warp-uniformly
       const OpDev* op = &args.ops[ti.kind == kEnd ? args.slots[0] : ti.slot];
+      if (ti.kind != kEnd && ti_need_ready && !wait_op_ready(c, lane, ti)) ti.kind = kEnd;
       int ok = 1;
       if (lane == 0) {
         // a claimed tile only ever waits on tiles that were claimed before it
@@ -356,36 +389,60 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (ti.kind == kEnd || !ok) break;
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
-      if (ti.kind == kCombine) continue;
 
-      // Weight tiles by tiled TMA.  The A operand of a down tile is the packed intermediate:
-      // consecutive rows, one TMA box (8, 32, 128 or 256 rows high, the smallest that holds the
-      // tile's rows); the A operand of a gate/up tile is gathered by the gather warps.
-      const bool g1 = ti.kind == kGateUp;
-      const CUtensorMap* tmw = g1 ? &op->tm_w1 : &op->tm_w2;
-      const int wrow0 = g1 ? ti.expert * 2 * args.I + ti.n * kTileN1 : ti.expert * args.H + ti.n * kTileN2;
-      const int wrow1 = g1 ? wrow0 + args.I : wrow0 + 128;
-      const int box = ti.rows <= 8 ? 8 : (ti.rows <= 32 ? 32 : (ti.rows <= 128 ? 128 : 256));
-      const CUtensorMap* tma = box == 8 ? &op->tm_a8 : (box == 32 ? &op->tm_a32 : (box == 128 ? &op->tm_a128 : &op->tm_a256));
-      const unsigned tx = (unsigned)kBBytes + (g1 ? 0u : (unsigned)(box * kRowBytes));
-      bool fail = false;
-      for (int kb = 0; kb < ti.kblocks; ++kb) {
-        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 5))) { fail = true; break; }
-        if (lane == 0) {
+      if (ti.kind != kCombine) {
+        // Weight tiles by tiled TMA.  The A operand of a down tile is the packed intermediate:
+        // consecutive rows, one TMA box (8, 32, 128 or 256 rows high, the smallest that holds
+        // the tile's rows); the A operand of a gate/up tile is gathered by the gather warps.
+        const bool g1 = ti.kind == kGateUp;
+        const CUtensorMap* tmw = g1 ? &op->tm_w1 : &op->tm_w2;
+        const int wrow0 = g1 ? ti.expert * 2 * args.I + ti.n * kTileN1 : ti.expert * args.H + ti.n * kTileN2;
+        const int wrow1 = g1 ? wrow0 + args.I : wrow0 + 128;
+        const int box = ti.rows <= 8 ? 8 : (ti.rows <= 32 ? 32 : (ti.rows <= 128 ? 128 : 256));
+        const CUtensorMap* tma = box == 8 ? &op->tm_a8 : (box == 32 ? &op->tm_a32 : (box == 128 ? &op->tm_a128 : &op->tm_a256));
+        const unsigned tx = (unsigned)kBBytes + (g1 ? 0u : (unsigned)(box * kRowBytes));
+        const int claim_at = min(kClaimAt, ti.kblocks - 1);
+        const int pf_at = max(claim_at, ti.kblocks - kPrefetchLead);
+        bool fail = false;
+        for (int kb = 0; kb < ti.kblocks; ++kb) {
+          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 5))) { fail = true; break; }
+          if (lane == 0) {
 #ifdef MOE_TIMING_PROBE
-          if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 0] = clock64();
+            if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 0] = clock64();
 #endif
-          unsigned char* sA = stages + (size_t)stage * kStageBytes;
-          unsigned char* sB = sA + kABytes;
-          mbar_expect_tx(&sc->full[stage], tx);
-          tma_tile_2d(sB, tmw, kb * kBlockK, wrow0, &sc->full[stage]);
-          tma_tile_2d(sB + kBHalfBytes, tmw, kb * kBlockK, wrow1, &sc->full[stage]);
-          if (!g1) tma_tile_2d(sA, tma, kb * kBlockK, ti.row0, &sc->full[stage]);
+            unsigned char* sA = stages + (size_t)stage * kStageBytes;
+            unsigned char* sB = sA + kABytes;
+            mbar_expect_tx(&sc->full[stage], tx);
+            tma_tile_2d(sB, tmw, kb * kBlockK, wrow0, &sc->full[stage]);
+            tma_tile_2d(sB + kBHalfBytes, tmw, kb * kBlockK, wrow1, &sc->full[stage]);
+            if (!g1) tma_tile_2d(sA, tma, kb * kBlockK, ti.row0, &sc->full[stage]);
+          }
+          __syncwarp();
+          if (++stage == kStages) { stage = 0; ph ^= 1u; }
+          if (kb == claim_at)              // claim ahead (never blocks here)
+            have_nx = claim_once(c, sc, rh, lane, nx, nx_need_ready) == 1;
+          if (kb == pf_at && have_nx && nx.kind != kCombine && lane < 3 * kAheadPrefetch) {
+            // shortly before the current tile ends, pull the first boxes of the next tile into L2
+            const OpDev* nop = &args.ops[nx.slot];
+            const bool n1 = nx.kind == kGateUp;
+            const int r0 = n1 ? nx.expert * 2 * args.I + nx.n * kTileN1 : nx.expert * args.H + nx.n * kTileN2;
+            const int r1 = n1 ? r0 + args.I : r0 + 128;
+            const int pk = lane / 3, which = lane % 3;
+            if (pk < nx.kblocks) {
+              if (which < 2) tma_prefetch_2d(n1 ? &nop->tm_w1 : &nop->tm_w2, pk * kBlockK, which ? r1 : r0);
+              else if (!n1) tma_prefetch_2d(nx.rows <= 128 ? &nop->tm_a128 : &nop->tm_a256, pk * kBlockK, nx.row0);
+            }
+          }
         }
-        __syncwarp();
-        if (++stage == kStages) { stage = 0; ph ^= 1u; }
+        if (fail) break;
       }
-      if (fail) break;
+      if (have_nx) {
+        ti = nx;
+        ti_need_ready = nx_need_ready;
+        have_nx = false;
+      } else {
+        claim_next(c, sc, rh, lane, ti, ti_need_ready);
+      }
     }
   } else if (warp == 1) {
     // ============================================================ MMA issuer
@@ -412,6 +469,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         const unsigned d0 = tmem + (use0 ? 0u : (unsigned)kAccCols);     // accumulator of rows 0..127
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
+#ifdef MOE_TIMING_PROBE
+          const long long t_fullB = clock64();
+#endif
           if (kind == kGateUp) {       // gathered rows arrive through their own barrier
             if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], (phA >> stage) & 1u, 12))) { fail = true; break; }
             phA ^= 1u << stage;
@@ -435,7 +495,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
             }
             tc_commit(&sc->empty[stage]);               // frees the stage when the MMAs retire
 #ifdef MOE_TIMING_PROBE
-            if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 3] = clock64();
+            if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 3] = t_fullB;
 #endif
           }
           __syncwarp();
