@@ -8,6 +8,8 @@
 namespace moe {
 
 // Tokens [t0, t1) by `nthr` cooperating threads (thread index tid); 8 bf16 per 16-byte access.
+// The k rows of a token are fetched eight at a time so that a thread keeps eight 16-byte
+// loads in flight; they are still ADDED in slot order j = 0..k-1.
 __device__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, int H, int tid,
                                       int nthr) {
   const int vec_per_row = H / 8;
@@ -21,16 +23,31 @@ __device__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, in
     float acc[8];
 #pragma unroll
     for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-    for (int j = 0; j < k; ++j) {
-      const int p = f2s[(size_t)t * k + j];
-      const float wj = w[(size_t)t * k + j];
-      const uint4 d = D[(size_t)p * vec_per_row + v];
-      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&d);
+    for (int j0 = 0; j0 < k; j0 += 8) {
+      float wj[8];
+      uint4 d[8];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float2 f = __bfloat1622float2(h[i]);
-        acc[2 * i] = fmaf(wj, f.x, acc[2 * i]);
-        acc[2 * i + 1] = fmaf(wj, f.y, acc[2 * i + 1]);
+      for (int i = 0; i < 8; ++i) {
+        const int j = j0 + i;
+        wj[i] = 0.f;
+        d[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (j < k) {
+          const int p = f2s[(size_t)t * k + j];
+          wj[i] = w[(size_t)t * k + j];
+          d[i] = D[(size_t)p * vec_per_row + v];
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) {
+        if (j0 + i < k) {
+          const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&d[i]);
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            const float2 f = __bfloat1622float2(h[c]);
+            acc[2 * c] = fmaf(wj[i], f.x, acc[2 * c]);
+            acc[2 * c + 1] = fmaf(wj[i], f.y, acc[2 * c + 1]);
+          }
+        }
       }
     }
     uint4 o;

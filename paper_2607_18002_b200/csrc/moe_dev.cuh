@@ -17,7 +17,7 @@ constexpr int kTileN2 = 256;         // output columns per down-GEMM tile
 constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kRowBytes = kBlockK * 2;
 constexpr int kStages = 3;           // shared-memory pipeline depth (64 KB per stage)
-constexpr int kCombineTokens = 32;   // tokens per combine tile
+constexpr int kCombineTokens = 16;   // tokens per combine tile
 constexpr int kPlanChunk = 256;      // routed rows ranked by one warp in the plan kernels
 constexpr int kGroupWork = 16;       // work tiles per dependency group of the tile list
 constexpr int kWorkRowsBf16 = 256;   // rows of a work tile: two m-tiles share each weight tile

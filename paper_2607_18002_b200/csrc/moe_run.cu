@@ -43,8 +43,7 @@ constexpr int kRing = 4;                               // tile-info ring depth
 constexpr int kAccCols = 256;                          // TMEM columns per accumulator
 constexpr int kEnd = -1;
 constexpr int kClaimAt = 2;                             // claim the next tile after this k-block
-constexpr int kAheadPrefetch = 3;                       // k-blocks of the next tile prefetched into L2
-constexpr int kPrefetchLead = 6;                        // ... this many k-blocks before the current tile ends
+constexpr int kPublishLead = 5;                         // try to hand the next tile on from this many k-blocks before the end
 
 struct TileInfo {
   int kind, slot, tile, m, row0, rows, n, kblocks, expert, cls;
@@ -365,6 +364,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     unsigned ph = 0, iph = 0;
     TileInfo ti, nx;
     bool ti_need_ready = false, nx_need_ready = false, have_nx = false;
+    bool ti_published = false, nx_published = false;
     ti.kind = kEnd;
     ti.slot = ti.tile = ti.m = ti.row0 = ti.rows = ti.n = ti.kblocks = ti.expert = ti.cls = 0;
     ti.t_claim = 0;
@@ -372,23 +372,27 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     claim_next(c, sc, rh, lane, ti, ti_need_ready);
     while (true) {
       ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);      // the claim loops exit warp-uniformly
-      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->iempty[islot], iph ^ 1u, 2))) break;
       const OpDev* op = &args.ops[ti.kind == kEnd ? args.slots[0] : ti.slot];
-      if (ti.kind != kEnd && ti_need_ready && !wait_op_ready(c, lane, ti)) ti.kind = kEnd;
-      int ok = 1;
-      if (lane == 0) {
-        // a claimed tile only ever waits on tiles that were claimed before it
-        if (ti.kind == kDown) ok = wait_counter(c, &op->g1_done[ti.m], args.I / kTileN1, 3);
-        if (ti.kind == kCombine) ok = wait_counter(c, &op->run->gemm_done, op->plan->n_gemm_tiles, 4);
-        if (!ok) ti.kind = kEnd;
-        fence_async_proxy();
-        sc->info[islot] = ti;
-        __threadfence_block();
-        mbar_arrive(&sc->ifull[islot]);
+      if (!ti_published) {
+        // blocking hand-off: a free ring slot, the op ready, the tile's dependencies met
+        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->iempty[islot], iph ^ 1u, 2))) break;
+        if (ti.kind != kEnd && ti_need_ready && !wait_op_ready(c, lane, ti)) ti.kind = kEnd;
+        int ok = 1;
+        if (lane == 0) {
+          // a claimed tile only ever waits on tiles that were claimed before it
+          if (ti.kind == kDown) ok = wait_counter(c, &op->g1_done[ti.m], args.I / kTileN1, 3);
+          if (ti.kind == kCombine) ok = wait_counter(c, &op->run->gemm_done, op->plan->n_gemm_tiles, 4);
+          if (!ok) ti.kind = kEnd;
+          fence_async_proxy();
+          sc->info[islot] = ti;
+          __threadfence_block();
+          mbar_arrive(&sc->ifull[islot]);
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
+        if (ti.kind == kEnd || !ok) break;
+        if (++islot == kRing) { islot = 0; iph ^= 1u; }
       }
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (ti.kind == kEnd || !ok) break;
-      if (++islot == kRing) { islot = 0; iph ^= 1u; }
+      ti_published = false;
 
       if (ti.kind != kCombine) {
         // Weight tiles by tiled TMA.  The A operand of a down tile is the packed intermediate:
@@ -402,7 +406,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         const CUtensorMap* tma = box == 8 ? &op->tm_a8 : (box == 32 ? &op->tm_a32 : (box == 128 ? &op->tm_a128 : &op->tm_a256));
         const unsigned tx = (unsigned)kBBytes + (g1 ? 0u : (unsigned)(box * kRowBytes));
         const int claim_at = min(kClaimAt, ti.kblocks - 1);
-        const int pf_at = max(claim_at, ti.kblocks - kPrefetchLead);
         bool fail = false;
         for (int kb = 0; kb < ti.kblocks; ++kb) {
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 5))) { fail = true; break; }
@@ -421,16 +424,29 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           if (++stage == kStages) { stage = 0; ph ^= 1u; }
           if (kb == claim_at)              // claim ahead (never blocks here)
             have_nx = claim_once(c, sc, rh, lane, nx, nx_need_ready) == 1;
-          if (kb == pf_at && have_nx && nx.kind != kCombine && lane < 3 * kAheadPrefetch) {
-            // shortly before the current tile ends, pull the first boxes of the next tile into L2
+          if (have_nx && !nx_published && kb > claim_at && kb >= ti.kblocks - kPublishLead) {
+            // Hand the next tile to the other warps before this one's last loads go out, if that
+            // takes no waiting: free ring slot, op ready, dependencies already met.
             const OpDev* nop = &args.ops[nx.slot];
-            const bool n1 = nx.kind == kGateUp;
-            const int r0 = n1 ? nx.expert * 2 * args.I + nx.n * kTileN1 : nx.expert * args.H + nx.n * kTileN2;
-            const int r1 = n1 ? r0 + args.I : r0 + 128;
-            const int pk = lane / 3, which = lane % 3;
-            if (pk < nx.kblocks) {
-              if (which < 2) tma_prefetch_2d(n1 ? &nop->tm_w1 : &nop->tm_w2, pk * kBlockK, which ? r1 : r0);
-              else if (!n1) tma_prefetch_2d(nx.rows <= 128 ? &nop->tm_a128 : &nop->tm_a256, pk * kBlockK, nx.row0);
+            bool can = __all_sync(0xffffffffu, mbar_try(&sc->iempty[islot], iph ^ 1u));
+            if (can && nx_need_ready) can = op_ready(&args, nop);
+            if (can) {
+              int met = 1;
+              if (lane == 0) {
+                if (nx.kind == kDown) met = ld_acquire(&nop->g1_done[nx.m]) >= args.I / kTileN1;
+                if (nx.kind == kCombine) met = ld_acquire(&nop->run->gemm_done) >= nop->plan->n_gemm_tiles;
+                if (met) {
+                  fence_async_proxy();
+                  sc->info[islot] = nx;
+                  __threadfence_block();
+                  mbar_arrive(&sc->ifull[islot]);
+                }
+              }
+              met = __shfl_sync(0xffffffffu, met, 0);
+              if (met) {
+                nx_published = true;
+                if (++islot == kRing) { islot = 0; iph ^= 1u; }
+              }
             }
           }
         }
@@ -439,7 +455,8 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (have_nx) {
         ti = nx;
         ti_need_ready = nx_need_ready;
-        have_nx = false;
+        ti_published = nx_published;
+        have_nx = nx_published = false;
       } else {
         claim_next(c, sc, rh, lane, ti, ti_need_ready);
       }
