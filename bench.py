@@ -33,7 +33,7 @@ METRIC = "moe_expert_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 KERNELS_PER_PLAN = 3          # histogram, scan + tile list, scatter
-DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c2s": (20, 3), "c3s": (10, 3)}
+DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c2s": (20, 3), "c3s": (10, 3)}
 
 
 def load_peaks():
@@ -124,10 +124,15 @@ class Workload:
         n_sets = 2 if self.spec.layers > 1 else 1          # c4 alternates two weight sets
         threads = os.cpu_count() or 8
         self.W_host = [synth.make_weights(self.spec, layer=i, threads=threads) for i in range(n_sets)]
-        self.W = [synth.Weights(w.w_gate_up.to(device), w.w_down.to(device)) for w in self.W_host]
+        dev = lambda t: None if t is None else t.to(device)
+        self.W = [synth.Weights(dev(w.w_gate_up), dev(w.w_down), dev(w.s_gate_up), dev(w.s_down))
+                  for w in self.W_host]
+        self.fp8 = sh.dtype == "fp8"
+        el = 1 if self.fp8 else 2
         self.layers = []
         self.ctx = moe.Context(sh.E, sh.k, sh.H, sh.I, max(T for _, T in self.spec.ops),
                                max_ops=len(self.spec.ops), tile_log_entries=tile_log,
+                               dtype=moe.MOE_DTYPE_FP8_E4M3 if self.fp8 else moe.MOE_DTYPE_BF16,
                                device=device)
         self.flops = 0.0
         self.bytes_alg = 0.0
@@ -142,17 +147,23 @@ class Workload:
                 hi = torch.from_numpy(op.ids).pin_memory()
                 hw = torch.from_numpy(op.w).pin_memory()
                 dx, di, dw = hx.to(device), hi.to(device), hw.to(device)
-                b = self.ctx.bind(op.cls, dx, di, dw, W.w_gate_up, W.w_down)
+                hs = None if op.x_scale is None else op.x_scale.pin_memory()
+                b = self.ctx.bind(op.cls, dx, di, dw, W.w_gate_up, W.w_down, x_scale=dev(hs),
+                                  s_gate_up=W.s_gate_up, s_down=W.s_down)
                 hy = torch.empty(b.y.shape, dtype=b.y.dtype).pin_memory()
                 bound.append(b)
-                host.append((hx, hi, hw, hy))
+                host.append((hx, hi, hw, hy, hs))
                 active[np.unique(op.ids)] = True
                 self.flops += 6.0 * op.ids.size * sh.H * sh.I
-                self.bytes_alg += 2 * op.T * sh.H * 2            # X once, y once
-                self.h2d += hx.numel() * 2 + hi.numel() * 4 + hw.numel() * 4
+                self.bytes_alg += op.T * sh.H * (el + 2)         # X once, y (bf16) once
+                if hs is not None:
+                    self.bytes_alg += hs.numel() * 4
+                self.h2d += hx.numel() * el + hi.numel() * 4 + hw.numel() * 4 + (0 if hs is None else hs.numel() * 4)
                 self.d2h += hy.numel() * 2
             # weights of the union of active experts of the launch, once
-            self.bytes_alg += float(active.sum()) * 3 * sh.H * sh.I * 2
+            self.bytes_alg += float(active.sum()) * 3 * sh.H * sh.I * el
+            if self.fp8:
+                self.bytes_alg += float(active.sum()) * 3 * (sh.H // 128) * (sh.I // 128) * 4
             self.layers.append((ops, bound, host))
         self.launches_per_step = sum(len(b) * KERNELS_PER_PLAN + 1 + (1 if self.spec.layers > 1 else 0)
                                      for _, b, _ in self.layers)
@@ -180,13 +191,15 @@ class Workload:
         for li, (_, bound, host) in enumerate(self.layers):
             if self.spec.layers > 1:
                 ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
-            for s, (b, (hx, hi, hw, hy)) in enumerate(zip(bound, host)):
+            for s, (b, (hx, hi, hw, hy, hs)) in enumerate(zip(bound, host)):
                 b.x.copy_(hx, non_blocking=True)
+                if hs is not None:
+                    b.x_scale.copy_(hs, non_blocking=True)
                 b.topk_ids.copy_(hi, non_blocking=True)
                 b.topk_w.copy_(hw, non_blocking=True)
                 ctx.plan(s, b)
             ctx.run(list(range(len(bound))), fuse_combine=True)
-            for b, (_, _, _, hy) in zip(bound, host):
+            for b, (_, _, _, hy, _) in zip(bound, host):
                 hy.copy_(b.y, non_blocking=True)
         torch.cuda.current_stream().synchronize()
 
@@ -199,7 +212,8 @@ def oracle_sample(w: Workload, seconds_target: float = 12.0):
     ops, _, _ = w.layers[0]
     op = max(ops, key=lambda o: o.T)
     Wh = w.W_host[0]
-    OW = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wh.w_gate_up, Wh.w_down)
+    OW = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wh.w_gate_up, Wh.w_down, Wh.s_gate_up, Wh.s_down)
+    rA = oracle.ROUND_E4M3_1X128 if sh.dtype == "fp8" else oracle.ROUND_NONE
     cores = oracle.threads()
     n, spent, done_tokens = max(2, cores // sh.k), 0.0, 0
     rng = np.random.default_rng(0)
@@ -207,7 +221,7 @@ def oracle_sample(w: Workload, seconds_target: float = 12.0):
         toks = rng.choice(op.T, size=min(n, op.T), replace=False).astype(np.int32)
         t0 = time.perf_counter()
         oracle.plan(op.ids, sh.E)
-        oracle.forward_tokens(OW, op.x, None, op.ids, op.w, toks)
+        oracle.forward_tokens(OW, op.x, op.x_scale, op.ids, op.w, toks, round_A=rA)
         dt = time.perf_counter() - t0
         spent += dt
         done_tokens, last_dt = len(toks), dt
@@ -299,7 +313,8 @@ def run_reference(args):
     sh = spec.shape
     Wh = synth.make_weights(spec, threads=os.cpu_count() or 8)
     op = max(synth.make_ops(spec), key=lambda o: o.T)
-    OW = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wh.w_gate_up, Wh.w_down)
+    OW = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wh.w_gate_up, Wh.w_down, Wh.s_gate_up, Wh.s_down)
+    rA = oracle.ROUND_E4M3_1X128 if sh.dtype == "fp8" else oracle.ROUND_NONE
     cores = oracle.threads()
     n_tok = max(4, (2 * cores) // sh.k)
     rng = np.random.default_rng(0)
@@ -308,7 +323,7 @@ def run_reference(args):
         toks = rng.choice(op.T, size=min(n_tok, op.T), replace=False).astype(np.int32)
         t0 = time.perf_counter()
         oracle.plan(op.ids, sh.E)
-        oracle.forward_tokens(OW, op.x, None, op.ids, op.w, toks)
+        oracle.forward_tokens(OW, op.x, op.x_scale, op.ids, op.w, toks, round_A=rA)
         dt = time.perf_counter() - t0
         if i >= args.warmup:
             times.append(dt)
@@ -379,20 +394,22 @@ def run_ours(args):
     t_run = float(np.mean(run_ms)) / 1e3
     flops_launch = w.flops / len(w.layers)
     bytes_launch = w.bytes_alg / len(w.layers)
-    tensor_frac = flops_launch / t_run / 1e12 / peaks["bf16_tflops"]
+    # the fp8 tensor peak is the measured bf16 peak x the nominal 2x ratio
+    tpeak = peaks["bf16_tflops"] * (2.0 if w.fp8 else 1.0)
+    tensor_frac = flops_launch / t_run / 1e12 / tpeak
     hbm_frac = bytes_launch / t_run / 1e9 / peaks["hbm_gbs"]
-    if args.workload == "c2":
+    if args.workload in ("c2", "c2s", "c5"):
         roof = {"bound": "hbm", "achieved": bytes_launch / t_run / 1e9, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": hbm_frac}
     else:
         roof = {"bound": "tensor", "achieved": flops_launch / t_run / 1e12,
-                "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": tensor_frac}
+                "peak": tpeak, "unit": "TFLOP/s", "frac": tensor_frac}
     roof.update({"traffic": None, "kernel": "moe_apk_kernel", "peak_source": peak_src,
                  "launch_ms_mean": 1e3 * t_run, "launch_ms_min": float(np.min(run_ms)),
                  "algorithmic_flops_per_launch": flops_launch,
                  "algorithmic_bytes_per_launch": bytes_launch,
                  "tensor_frac_of_burst": tensor_frac,
-                 "tensor_frac_of_sustained": flops_launch / t_run / 1e12 / peaks["bf16_tflops_sustained"],
+                 "tensor_frac_of_sustained": flops_launch / t_run / 1e12 / (peaks["bf16_tflops_sustained"] * (2.0 if w.fp8 else 1.0)),
                  "hbm_frac": hbm_frac})
 
     tiles = tile_stats(w) if args.tile_log else None
@@ -407,7 +424,8 @@ def run_ours(args):
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
             "warmup": Wm, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3" if w.fp8 else "bf16",
+            "data": "synthetic",
             "config": {"workload": args.workload, "ops": [[c, t] for c, t in w.spec.ops],
                        "layers": w.spec.layers, "experts": sh.E, "top_k": sh.k, "hidden": sh.H,
                        "inter": sh.I, "l2": "inputs_exceed_l2 (weights >> 126 MB, no flush)",
@@ -425,7 +443,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c2s", "c3s"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "c2s", "c3s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tile-log", action="store_true", help="add per-tile timing statistics of one extra untimed step")

@@ -21,6 +21,7 @@ constexpr int kCombineTokens = 16;   // tokens per combine tile
 constexpr int kPlanChunk = 256;      // routed rows ranked by one warp in the plan kernels
 constexpr int kGroupWork = 16;       // work tiles per dependency group of the tile list
 constexpr int kWorkRowsBf16 = 256;   // rows of a work tile: two m-tiles share each weight tile
+constexpr int kWorkRowsFp8 = 128;    // fp8: the accumulator and both partial buffers fill TMEM
 constexpr int kMaxOps = 16;
 constexpr int kMaxExperts = 1024;
 
@@ -79,7 +80,8 @@ struct __align__(128) OpDev {
   const unsigned* ready;
   unsigned* done;
   // workspace-owned
-  __nv_bfloat16* A;      // [Rmax, I]  SwiGLU output, packed order
+  __nv_bfloat16* A;      // [Rmax, I]  SwiGLU output, packed order (e4m3 bytes in the fp8 path)
+  float* a_scale;        // [Rmax, I/128] fp32 scales of A (fp8 path)
   __nv_bfloat16* D;      // [Rmax, H]  expert output, packed order
   MTile* mtiles;         // [max_mtiles]
   int4* tile_list;       // [max_tiles] queue entries in claim order
@@ -118,6 +120,7 @@ struct RunArgs {
   int n_ops;
   int fuse_combine;
   int E, k, H, I;
+  int dtype, kb_elems;    // MOE_DTYPE_*; K elements per pipeline stage (64 bf16 / 128 e4m3)
 #ifdef MOE_TIMING_PROBE
   long long* dbg;
 #endif

@@ -38,7 +38,7 @@ int check_config(const moe_config_t* c) {
   if (c->top_k < 1 || c->top_k > 32 || c->top_k > c->n_experts) return MOE_EINVAL;
   if (c->hidden < kTileN2 || c->hidden % kTileN2) return MOE_EINVAL;
   if (c->inter < kTileN1 || c->inter % kTileN1) return MOE_EINVAL;
-  if (c->dtype != MOE_DTYPE_BF16) return MOE_EINVAL;
+  if (c->dtype != MOE_DTYPE_BF16 && c->dtype != MOE_DTYPE_FP8_E4M3) return MOE_EINVAL;
   if (c->max_tokens_per_op < 1 || c->max_ops < 1 || c->max_ops > kMaxOps) return MOE_EINVAL;
   if ((long long)c->max_tokens_per_op * c->top_k > (1 << 20) * (long long)kTileM) return MOE_EINVAL;
   if (c->wait_limit_us < 0 || c->tile_log_entries < 0 || c->n_ctas < 0) return MOE_EINVAL;
@@ -102,15 +102,18 @@ struct moe_ctx {
 
 namespace {
 
-// 2-D bf16 tensor map: `rows` x `cols` row-major, box = box_rows x kBlockK columns, swizzle
+// 2-D tensor map (bf16, or e4m3 bytes): `rows` x `cols` row-major, box = box_rows x kBlockK columns, swizzle
 // as wide as a box row
 int make_map(moe_ctx* ctx, CUtensorMap* out, const void* base, size_t rows, size_t cols,
              int box_rows) {
+  const bool fp8 = ctx->cfg.dtype == MOE_DTYPE_FP8_E4M3;
+  const size_t el = fp8 ? 1 : 2;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  cuuint32_t box[2] = {(cuuint32_t)kBlockK, (cuuint32_t)box_rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * el};
+  cuuint32_t box[2] = {(cuuint32_t)(kRowBytes / el), (cuuint32_t)box_rows};   // 128 bytes per box row
   cuuint32_t estr[2] = {1, 1};
-  CUresult r = ctx->encode(out, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims,
+  CUresult r = ctx->encode(out, fp8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2,
+                           const_cast<void*>(base), dims,
                            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            kRowBytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
@@ -198,6 +201,8 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   if (op->after_op < -1 || op->after_op >= c.max_ops || op->after_op == slot) return MOE_EINVAL;
   if (!op->counts || !op->offsets) return MOE_EINVAL;
   if (!op->w_gate_up || !op->w_down || !aligned16(op->w_gate_up) || !aligned16(op->w_down)) return MOE_EINVAL;
+  if (c.dtype == MOE_DTYPE_FP8_E4M3 && (!op->s_gate_up || !op->s_down || (op->n_tokens > 0 && !op->x_scale)))
+    return MOE_EINVAL;
   if (op->n_tokens > 0) {
     if (!op->x || !op->topk_ids || !op->topk_w || !op->y || !op->sorted_to_flat || !op->flat_to_sorted)
       return MOE_EINVAL;
@@ -217,6 +222,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   h.sorted_to_flat = op->sorted_to_flat; h.flat_to_sorted = op->flat_to_sorted;
   h.ready = op->ready; h.done = op->done;
   h.A = reinterpret_cast<__nv_bfloat16*>(sb + L.A_off);
+  h.a_scale = reinterpret_cast<float*>(sb + L.A_off + align_up((size_t)L.max_rows * c.inter, 16));
   h.D = reinterpret_cast<__nv_bfloat16*>(sb + L.D_off);
   h.mtiles = reinterpret_cast<MTile*>(sb + L.mtiles_off);
   h.tile_list = reinterpret_cast<int4*>(sb + L.tiles_off);
@@ -238,7 +244,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   if (cudaMemcpyAsync(ctx->op_dev(slot), &h, sizeof(h), cudaMemcpyHostToDevice, st) != cudaSuccess)
     return MOE_ECUDA;
   if (launch_plan(ctx->op_dev(slot), ctx->g(), slot, op->n_tokens, c.top_k, c.n_experts, L.NT1, L.NT2,
-                  kWorkRowsBf16, st) != cudaSuccess)
+                  c.dtype == MOE_DTYPE_FP8_E4M3 ? kWorkRowsFp8 : kWorkRowsBf16, st) != cudaSuccess)
     return MOE_ECUDA;
   ctx->ops[slot] = *op;
   ctx->planned[slot] = true;
@@ -271,6 +277,8 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
   a.n_ops = n_ops;
   a.fuse_combine = fuse_combine ? 1 : 0;
   a.E = c.n_experts; a.k = c.top_k; a.H = c.hidden; a.I = c.inter;
+  a.dtype = c.dtype;
+  a.kb_elems = c.dtype == MOE_DTYPE_FP8_E4M3 ? 128 : kBlockK;
   a.wait_ns = (long long)c.wait_limit_us * 1000;
 #ifdef MOE_TIMING_PROBE
   a.dbg = reinterpret_cast<long long*>(ctx->ws + ctx->L.log_off);   // the tile log area doubles as probe buffer

@@ -29,6 +29,7 @@
 // kernel records MOE_ETIMEOUT, raises the abort word, and all CTAs drain and return.
 #include "moe_combine.cuh"
 #include "moe_ptx.cuh"
+#include <cuda_fp8.h>
 
 namespace moe {
 
@@ -53,6 +54,9 @@ struct TileInfo {
 struct SharedCtl {
   unsigned long long full[kStages], fullA[kStages], empty[kStages];
   unsigned long long tfull[2], tempty[2];
+  unsigned long long pfull[2], pempty[2];          // fp8: per-k-block partial products (two column halves)
+  unsigned long long xbar[4];                      // fp8: amax exchange between the two warps of a quadrant
+  float amax_x[2][4][32];
   unsigned long long ifull[kRing], iempty[kRing], done[kRing];
   TileInfo info[kRing];
   unsigned tmem_base;
@@ -175,7 +179,7 @@ __device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, in
   ti.slot = slot;
   ti.tile = (int)local;
   ti.cls = cls;
-  ti.kblocks = ti.kind == kCombine ? 0 : (ti.kind == kGateUp ? a->H : a->I) / kBlockK;
+  ti.kblocks = ti.kind == kCombine ? 0 : (ti.kind == kGateUp ? a->H : a->I) / a->kb_elems;
   return 1;
 }
 
@@ -301,6 +305,137 @@ __device__ __forceinline__ float silu_mul(float g, float u) {
   return fmaf(hg, t, hg) * u;                     // g * sigmoid(g) = g/2 * (1 + tanh(g/2))
 }
 
+// ------------------------------------------------------------------ FP8 (e4m3, fp32 block scales)
+constexpr unsigned kPartialCol = 256;     // TMEM: columns 0..255 fp32 accumulator, 256..511 two partial halves
+// instruction descriptor: D fp32, A/B e4m3, both K-major, M = 128, N = 128
+constexpr unsigned kIdescF8 = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+
+// One e4m3 tile on the epilogue warps.  Thread = (accumulator row, 64-column slice of each
+// 128-column half).  Per k-block and half: partial * (activation scale of the row and k-block
+// * weight scale of the half and k-block) is added into the accumulator columns.  Then
+// gate/up tiles apply SwiGLU and re-quantise the 128 outputs of the row to e4m3 with one
+// fp32 scale (amax / 448) -- the one quantisation on the path -- and down tiles store bf16.
+__device__ inline bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev* op, const TileInfo& ti,
+                                    unsigned tmem, int warp, int lane, unsigned (&eph)[2],
+                                    unsigned& xph) {
+  const RunArgs& a = *c.a;
+  const int q = warp & 3, ch = (warp - 8) >> 2;
+  const int row = q * 32 + lane;
+  const bool valid = row < ti.rows;
+  const bool g1 = ti.kind == kGateUp;
+  const int HB = a.H / 128, IB = a.I / 128;
+  const unsigned lane_addr = tmem + ((unsigned)(q * 32) << 16);
+  // scale streams of this row / tile
+  const float* sx;
+  const float *sw0, *sw1;
+  if (g1) {
+    const int tok = valid ? op->sorted_to_flat[ti.row0 + row] / a.k : 0;
+    sx = op->x_scale + (size_t)tok * HB;
+    sw0 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + ti.n) * HB;
+    sw1 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + IB + ti.n) * HB;
+  } else {
+    sx = op->a_scale + (size_t)(ti.row0 + (valid ? row : 0)) * IB;
+    sw0 = op->s_down + ((size_t)ti.expert * HB + 2 * ti.n) * IB;
+    sw1 = sw0 + IB;
+  }
+  float fx = sx[0], f0 = sw0[0], f1 = sw1[0];
+  for (int kb = 0; kb < ti.kblocks; ++kb) {
+    float nfx = 0.f, nf0 = 0.f, nf1 = 0.f;
+    if (kb + 1 < ti.kblocks) { nfx = sx[kb + 1]; nf0 = sw0[kb + 1]; nf1 = sw1[kb + 1]; }
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->pfull[h], eph[h], 19))) return false;
+      eph[h] ^= 1u;
+      tc_fence_after();
+      const float s = fx * (h ? f1 : f0);
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        const unsigned col = (unsigned)(h * 128 + ch * 64 + cc * 32);
+        unsigned p[32], acc[32];
+        tc_ld32(lane_addr + kPartialCol + col, p);
+        if (kb > 0) tc_ld32(lane_addr + col, acc);
+        tc_wait_ld();
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          const float v = __uint_as_float(p[i]) * s;
+          acc[i] = __float_as_uint(kb > 0 ? v + __uint_as_float(acc[i]) : v);
+        }
+        tc_st32(lane_addr + col, acc);
+      }
+      tc_wait_st();
+      tc_fence_before();
+      mbar_arrive(&sc->pempty[h]);                // the partial buffer may be overwritten
+    }
+    fx = nfx; f0 = nf0; f1 = nf1;
+  }
+  // the accumulator is complete
+  if (g1) {
+    float o[64];
+    float amax = 0.f;
+#pragma unroll
+    for (int cc = 0; cc < 2; ++cc) {
+      unsigned g[32], u[32];
+      tc_ld32(lane_addr + (unsigned)(ch * 64 + cc * 32), g);
+      tc_ld32(lane_addr + 128u + (unsigned)(ch * 64 + cc * 32), u);
+      tc_wait_ld();
+#pragma unroll
+      for (int i = 0; i < 32; ++i) {
+        const float gv = __uint_as_float(g[i]);
+        const float v = __fdividef(gv, 1.0f + __expf(-gv)) * __uint_as_float(u[i]);
+        o[cc * 32 + i] = v;
+        amax = fmaxf(amax, fabsf(v));
+      }
+    }
+    // the row's 128 outputs live in two threads (ch = 0, 1): exchange the partial maxima
+    sc->amax_x[ch][q][lane] = amax;
+    mbar_arrive(&sc->xbar[q]);
+    if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->xbar[q], xph, 20))) return false;
+    xph ^= 1u;
+    amax = fmaxf(amax, sc->amax_x[ch ^ 1][q][lane]);
+    const float scale = amax > 0.f ? amax / 448.0f : 1.0f;
+    const float inv = amax > 0.f ? 448.0f / amax : 0.0f;
+    if (valid) {
+      unsigned char* dst = static_cast<unsigned char*>((void*)op->A) + (size_t)(ti.row0 + row) * a.I +
+                           (size_t)ti.n * 128 + ch * 64;
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        unsigned w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const float* v = o + j * 16 + i * 4;
+          const unsigned lo = __nv_cvt_float2_to_fp8x2(make_float2(v[0] * inv, v[1] * inv), __NV_SATFINITE, __NV_E4M3);
+          const unsigned hi = __nv_cvt_float2_to_fp8x2(make_float2(v[2] * inv, v[3] * inv), __NV_SATFINITE, __NV_E4M3);
+          w[i] = lo | (hi << 16);
+        }
+        reinterpret_cast<uint4*>(dst)[j] = make_uint4(w[0], w[1], w[2], w[3]);
+      }
+      if (ch == 0) op->a_scale[(size_t)(ti.row0 + row) * IB + ti.n] = scale;
+    }
+  } else {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        unsigned v[32];
+        tc_ld32(lane_addr + (unsigned)(h * 128 + ch * 64 + cc * 32), v);
+        tc_wait_ld();
+        if (valid) {
+          __nv_bfloat16* dst = op->D + (size_t)(ti.row0 + row) * a.H + (size_t)ti.n * kTileN2 + h * 128 + ch * 64 + cc * 32;
+          uint4 o4[4];
+          __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(o4);
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            oh[i] = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+#pragma unroll
+          for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(dst)[i] = o4[i];
+        }
+      }
+    }
+  }
+  tc_fence_before();
+  return true;
+}
+
 // ------------------------------------------------------------------ the persistent kernel
 // which accumulator(s) a tile uses: a tile of up to 128 rows alternates between the two, a
 // tile of up to 256 rows takes both (rows 0..127 -> accumulator 0, rows 128..255 -> 1).
@@ -313,8 +448,11 @@ struct AccUse {
   }
 };
 
+template <bool kFp8>
 __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_constant__ RunArgs args,
                                                               RunHead* rh) {
+  constexpr int kKb = kFp8 ? 128 : kBlockK;     // K elements per stage (128 bytes per row either way)
+  constexpr int kEl = kFp8 ? 1 : 2;             // bytes per element
   extern __shared__ unsigned char smem_raw[];
   unsigned char* stages = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -328,7 +466,13 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       mbar_init(&sc->fullA[s], kGatherThreads);
       mbar_init(&sc->empty[s], 1);
     }
-    for (int s = 0; s < 2; ++s) { mbar_init(&sc->tfull[s], 1); mbar_init(&sc->tempty[s], 256); }
+    for (int s = 0; s < 2; ++s) {
+      mbar_init(&sc->tfull[s], 1);
+      mbar_init(&sc->tempty[s], 256);
+      mbar_init(&sc->pfull[s], 1);
+      mbar_init(&sc->pempty[s], 256);
+    }
+    for (int s = 0; s < 4; ++s) mbar_init(&sc->xbar[s], 64);
     // a ring slot is released by the MMA warp, the committer and each gather warp
     for (int s = 0; s < kRing; ++s) {
       mbar_init(&sc->ifull[s], 1);
@@ -416,9 +560,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
             unsigned char* sA = stages + (size_t)stage * kStageBytes;
             unsigned char* sB = sA + kABytes;
             mbar_expect_tx(&sc->full[stage], tx);
-            tma_tile_2d(sB, tmw, kb * kBlockK, wrow0, &sc->full[stage]);
-            tma_tile_2d(sB + kBHalfBytes, tmw, kb * kBlockK, wrow1, &sc->full[stage]);
-            if (!g1) tma_tile_2d(sA, tma, kb * kBlockK, ti.row0, &sc->full[stage]);
+            tma_tile_2d(sB, tmw, kb * kKb, wrow0, &sc->full[stage]);
+            tma_tile_2d(sB + kBHalfBytes, tmw, kb * kKb, wrow1, &sc->full[stage]);
+            if (!g1) tma_tile_2d(sA, tma, kb * kKb, ti.row0, &sc->full[stage]);
           }
           __syncwarp();
           if (++stage == kStages) { stage = 0; ph ^= 1u; }
@@ -467,7 +611,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     int dbg_i = 0;
 #endif
     int stage = 0, islot = 0;
-    unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0;
+    unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0, pph[2] = {0, 0};
     AccUse accs;
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 6))) break;
@@ -476,7 +620,39 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       const int rows = sc->info[islot].rows;
       if (kind == kEnd) break;
       bool fail = false;
-      if (kind != kCombine) {
+      if (kFp8 && kind != kCombine) {
+        // FP8 with fp32 block scales: the tensor core cannot apply a scale per 128-deep K block,
+        // so every k-block (= one scale block) is multiplied into a FRESH partial buffer, one
+        // per 128-column half of the weight tile (each half has a single weight scale), and the
+        // epilogue warps scale-and-add it into the fp32 accumulator columns of TMEM.
+        for (int kb = 0; kb < kblocks; ++kb) {
+          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
+          if (kind == kGateUp) {
+            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], (phA >> stage) & 1u, 12))) { fail = true; break; }
+            phA ^= 1u << stage;
+          }
+          for (int h = 0; h < 2 && !fail; ++h) {
+            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->pempty[h], pph[h] ^ 1u, 18))) { fail = true; break; }
+            pph[h] ^= 1u;
+            tc_fence_after();
+            if (lane == 0) {
+              fence_async_proxy_smem();
+              const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
+              const unsigned long long ad = umma_desc(sA, kRowBytes);
+              const unsigned long long bd = umma_desc(sA + kABytes + h * kBHalfBytes, kRowBytes);
+#pragma unroll
+              for (int k4 = 0; k4 < 4; ++k4)            // 32 e4m3 elements (32 bytes) per step
+                tc_mma_f8(tmem + kPartialCol + (unsigned)h * 128u, ad + 2ull * k4, bd + 2ull * k4, kIdescF8, k4 ? 1u : 0u);
+              tc_commit(&sc->pfull[h]);
+              if (h == 1) tc_commit(&sc->empty[stage]);
+            }
+            __syncwarp();
+          }
+          if (fail) break;
+          if (++stage == kStages) { stage = 0; ph ^= 1u; }
+        }
+        if (fail) break;
+      } else if (kind != kCombine) {
         bool use0, use1;
         accs.take(rows, use0, use1);
         if (use0 && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[0], aph[0] ^ 1u, 7))) break;
@@ -565,7 +741,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       }
       const OpDev* op = &args.ops[slot];
       const unsigned char* X = static_cast<const unsigned char*>(op->x) + chunk * 16;
-      const size_t pitch = (size_t)args.H * 2;
+      const size_t pitch = (size_t)args.H * kEl;
       int tok[kPasses];
 #pragma unroll
       for (int j = 0; j < kPasses; ++j) {
@@ -578,7 +754,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         const unsigned ph = (kiter / kStages) & 1u;
         if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 14))) { fail = true; break; }
         const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
-        const unsigned char* Xk = X + (size_t)kb * (kBlockK * 2);
+        const unsigned char* Xk = X + (size_t)kb * kRowBytes;
 #pragma unroll
         for (int j = 0; j < kPasses; ++j) {
           const int r = rbase + kRowsPerPass * j;
@@ -620,7 +796,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     const int half = (warp - 8) >> 2;             // which half of the columns
     const int etid = threadIdx.x - 256;           // 0..255
     int islot = 0;
-    unsigned iph = 0, aph[2] = {0, 0};
+    unsigned iph = 0, aph[2] = {0, 0}, eph[2] = {0, 0}, xph = 0;
     AccUse accs;
     unsigned char* scratch = sc->epi_scratch[warp - 8];
     const int srow = lane >> 2, schunk = lane & 3;          // this lane's part of a store
@@ -632,6 +808,8 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       bool ok = true;
       if (ti.kind == kCombine) {
         combine_tokens(op, ti.row0, ti.row0 + ti.rows, args.k, args.H, etid, 256);
+      } else if (kFp8) {
+        ok = epilogue_fp8(c, sc, op, ti, tmem, warp, lane, eph, xph);
       } else {
         bool use[2];
         accs.take(ti.rows, use[0], use[1]);
@@ -716,12 +894,16 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 }
 
 cudaError_t prepare_run_kernel() {
-  return cudaFuncSetAttribute(moe_apk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(moe_apk_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       (int)kSmemBytes);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(moe_apk_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                               (int)kSmemBytes);
 }
 
 cudaError_t launch_run(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream) {
-  moe_apk_kernel<<<n_ctas, kThreads, kSmemBytes, stream>>>(args, rh);
+  if (args.dtype == MOE_DTYPE_FP8_E4M3) moe_apk_kernel<true><<<n_ctas, kThreads, kSmemBytes, stream>>>(args, rh);
+  else moe_apk_kernel<false><<<n_ctas, kThreads, kSmemBytes, stream>>>(args, rh);
   return cudaGetLastError();
 }
 

@@ -1,0 +1,93 @@
+"""GPU parity of the FP8 e4m3 block-scaled path against the oracle on the same stored bytes.
+
+The oracle consumes code * scale exactly and mirrors the one quantisation that is part of
+the encoding (the SwiGLU output to e4m3 with one fp32 scale per row and 128 columns);
+acceptance is |gpu - ref| <= 4e-2 + 4e-2 |ref| elementwise plus a relative-L2 bound of 3e-2.
+The un-mirrored oracle (no rounding of the intermediate) is reported for information."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2607_18002_b200 as moe
+from workloads import synth
+
+from gpu_util import (ATOL8, REL_L2_8, RTOL8, assert_close, bind_ops, check_plan, make_ctx,
+                      oracle_weights, weights_to)
+
+pytestmark = pytest.mark.gpu
+
+
+def _run(spec, ops=None, W=None, budget=None):
+    W = W or synth.make_weights(spec)
+    ops = ops or synth.make_ops(spec)
+    ctx = make_ctx(spec, max_tokens=max(o.T for o in ops), max_ops=len(ops))
+    bound = bind_ops(ctx, ops, weights_to(W))
+    if budget is not None:
+        ctx.set_budget(budget)
+    for s, b in enumerate(bound):
+        ctx.plan(s, b)
+    ctx.run(list(range(len(bound))), fuse_combine=True)
+    ctx.check()
+    return ctx, bound, ops, W
+
+
+@pytest.mark.parametrize("shape", [synth.Shape(8, 2, 256, 128, "fp8"), synth.Shape(8, 2, 512, 256, "fp8"),
+                                   synth.Shape(16, 4, 768, 384, "fp8")], ids=["h256", "h512", "h768"])
+def test_small_fp8_matches_mirrored_oracle(shape):
+    spec = synth.Spec("fp8s", shape, ((synth.PREFILL, 300), (synth.DECODE, 37)), "softmax_topk",
+                      None, 1.0, -1.0, 31)
+    ctx, bound, ops, W = _run(spec)
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        check_plan(b, op, shape.E)
+        ref = oracle.forward(OW, op.x, op.x_scale, op.ids, op.w, round_A=oracle.ROUND_E4M3_1X128)
+        got = b.y.float().cpu().numpy()
+        assert_close(got, ref["y"], atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
+        plain = oracle.forward(OW, op.x, op.x_scale, op.ids, op.w)["y"]
+        rel = np.linalg.norm(got - plain) / np.linalg.norm(plain)
+        assert rel < 8e-2, rel          # information: distance to the un-mirrored reference
+
+
+def test_fp8_schedule_independence_bitwise():
+    spec = synth.Spec("fp8s", synth.Shape(8, 2, 512, 256, "fp8"), ((synth.PREFILL, 300), (synth.DECODE, 37)),
+                      "softmax_topk", None, 1.0, -1.0, 32)
+    W = synth.make_weights(spec)
+    ops = synth.make_ops(spec)
+    outs = []
+    for budget in (0, 16, 1000):
+        _, bound, _, _ = _run(spec, ops=ops, W=W, budget=budget)
+        outs.append([b.y.clone() for b in bound])
+    for o in outs[1:]:
+        for a, b in zip(outs[0], o):
+            assert torch.equal(a, b)
+
+
+def test_fp8_requires_scales():
+    spec = synth.Spec("fp8s", synth.Shape(8, 2, 256, 128, "fp8"), ((synth.PREFILL, 16),), "softmax_topk",
+                      None, 1.0, -1.0, 33)
+    W = weights_to(synth.make_weights(spec))
+    op = synth.make_ops(spec)[0]
+    ctx = make_ctx(spec)
+    b = ctx.bind(op.cls, op.x.cuda(), torch.from_numpy(op.ids).cuda(), torch.from_numpy(op.w).cuda(),
+                 W.w_gate_up, W.w_down)          # no scales
+    with pytest.raises(moe.MoeError) as ei:
+        ctx.plan(0, b)
+    assert ei.value.code == moe.MOE_EINVAL
+
+
+def test_c5_full_size_sampled():
+    """C5 in the launch configuration the bench times (4096 prefill + 512 decode tokens, one
+    persistent launch); the oracle evaluates a seeded token sample of each op."""
+    spec = synth.SPECS["c5"]
+    W = synth.make_weights(spec, threads=16)
+    ctx, bound, ops, _ = _run(spec, W=W, budget=32)
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        check_plan(b, op, spec.shape.E)
+        toks = np.random.default_rng(5).choice(op.T, size=48, replace=False).astype(np.int32)
+        ref = oracle.forward_tokens(OW, op.x, op.x_scale, op.ids, op.w, toks,
+                                    round_A=oracle.ROUND_E4M3_1X128)
+        got = b.y[torch.from_numpy(toks).long().cuda()].float().cpu().numpy()
+        assert_close(got, ref, atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
+        assert torch.isfinite(b.y.float()).all()
