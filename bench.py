@@ -33,7 +33,7 @@ METRIC = "moe_expert_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 KERNELS_PER_PLAN = 3          # histogram, scan + tile list, scatter
-DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c2s": (20, 3), "c3s": (10, 3)}
+DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c2s": (20, 3), "c3s": (10, 3), "c5s": (10, 3)}
 
 
 def load_peaks():
@@ -398,7 +398,7 @@ def run_ours(args):
     tpeak = peaks["bf16_tflops"] * (2.0 if w.fp8 else 1.0)
     tensor_frac = flops_launch / t_run / 1e12 / tpeak
     hbm_frac = bytes_launch / t_run / 1e9 / peaks["hbm_gbs"]
-    if args.workload in ("c2", "c2s", "c5"):
+    if args.workload in ("c2", "c2s", "c5", "c5s"):
         roof = {"bound": "hbm", "achieved": bytes_launch / t_run / 1e9, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": hbm_frac}
     else:
@@ -443,7 +443,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "c2s", "c3s"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "c2s", "c3s", "c5s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tile-log", action="store_true", help="add per-tile timing statistics of one extra untimed step")

@@ -52,9 +52,9 @@ struct TileInfo {
 };
 
 struct SharedCtl {
-  unsigned long long full[kStages], fullA[kStages], empty[kStages];
+  unsigned long long full[kStages], fullA[kStages], empty[kStages], emptyA[kStages];
   unsigned long long tfull[2], tempty[2];
-  unsigned long long pfull[2], pempty[2];          // fp8: per-k-block partial products (two column halves)
+  unsigned long long pfull[4], pempty[4];          // fp8: per-k-block partial products: [column half][2 buffers]
   unsigned long long xbar[4];                      // fp8: amax exchange between the two warps of a quadrant
   float amax_x[2][4][32];
   unsigned long long ifull[kRing], iempty[kRing], done[kRing];
@@ -96,6 +96,28 @@ __device__ __noinline__ bool mbar_wait_slow(const Ctx& c, void* bar, unsigned pa
 __device__ __forceinline__ bool mbar_wait(const Ctx& c, void* bar, unsigned parity, int where) {
   if (mbar_try(bar, parity)) return true;
   return mbar_wait_slow(c, bar, parity, where);
+}
+
+// the same wait without any function call: for code that keeps many registers live across it
+__device__ __forceinline__ bool mbar_wait_inline(const Ctx& c, void* bar, unsigned parity, int where) {
+  unsigned long long t0 = 0;
+  for (unsigned it = 0;; ++it) {
+    if (mbar_try(bar, parity)) return true;
+    if ((it & 63u) == 63u) {
+      if (aborted(c)) return false;
+      const unsigned long long now = gtime_ns();
+      if (t0 == 0) t0 = now;
+      else if ((long long)(now - t0) > c.a->wait_ns) {
+        if (atomicCAS(&c.st->code, 0, MOE_ETIMEOUT) == 0) {
+          c.st->detail[0] = where; c.st->detail[1] = (int)blockIdx.x;
+          c.st->detail[2] = (int)threadIdx.x; c.st->detail[3] = (int)parity;
+        }
+        __threadfence();
+        atomicExch(&c.st->abort, 1);
+        return false;
+      }
+    }
+  }
 }
 
 // spin until *p >= target (acquire); one thread
@@ -306,18 +328,18 @@ __device__ __forceinline__ float silu_mul(float g, float u) {
 }
 
 // ------------------------------------------------------------------ FP8 (e4m3, fp32 block scales)
-constexpr unsigned kPartialCol = 256;     // TMEM: columns 0..255 fp32 accumulator, 256..511 two partial halves
 // instruction descriptor: D fp32, A/B e4m3, both K-major, M = 128, N = 128
 constexpr unsigned kIdescF8 = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
 
 // One e4m3 tile on the epilogue warps.  Thread = (accumulator row, 64-column slice of each
-// 128-column half).  Per k-block and half: partial * (activation scale of the row and k-block
-// * weight scale of the half and k-block) is added into the accumulator columns.  Then
-// gate/up tiles apply SwiGLU and re-quantise the 128 outputs of the row to e4m3 with one
-// fp32 scale (amax / 448) -- the one quantisation on the path -- and down tiles store bf16.
-__device__ inline bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev* op, const TileInfo& ti,
-                                    unsigned tmem, int warp, int lane, unsigned (&eph)[2],
-                                    unsigned& xph) {
+// 128-column half); its 128 fp32 accumulators stay in registers (the epilogue warps raise
+// their register allowance for this).  Per k-block and half: partial * (activation scale of
+// the row and k-block * weight scale of the half and k-block) is added in.  Then gate/up
+// tiles apply SwiGLU and re-quantise the 128 outputs of the row to e4m3 with one fp32 scale
+// (amax / 448) -- the one quantisation on the path -- and down tiles store bf16.
+__device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev* op, const TileInfo& ti,
+                                             unsigned tmem, int warp, int lane, unsigned& eph,
+                                             unsigned& xph) {
   const RunArgs& a = *c.a;
   const int q = warp & 3, ch = (warp - 8) >> 2;
   const int row = q * 32 + lane;
@@ -338,58 +360,49 @@ __device__ inline bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev* op, cons
     sw0 = op->s_down + ((size_t)ti.expert * HB + 2 * ti.n) * IB;
     sw1 = sw0 + IB;
   }
+  float acc[128];                                 // [half][64]
+#pragma unroll
+  for (int i = 0; i < 128; ++i) acc[i] = 0.f;
   float fx = sx[0], f0 = sw0[0], f1 = sw1[0];
   for (int kb = 0; kb < ti.kblocks; ++kb) {
     float nfx = 0.f, nf0 = 0.f, nf1 = 0.f;
     if (kb + 1 < ti.kblocks) { nfx = sx[kb + 1]; nf0 = sw0[kb + 1]; nf1 = sw1[kb + 1]; }
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
-      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->pfull[h], eph[h], 19))) return false;
-      eph[h] ^= 1u;
+      const int pb = h * 2 + (kb & 1);
+      if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->pfull[pb], (eph >> pb) & 1u, 19))) return false;
+      eph ^= 1u << pb;
+
       tc_fence_after();
       const float s = fx * (h ? f1 : f0);
 #pragma unroll
       for (int cc = 0; cc < 2; ++cc) {
-        const unsigned col = (unsigned)(h * 128 + ch * 64 + cc * 32);
-        unsigned p[32], acc[32];
-        tc_ld32(lane_addr + kPartialCol + col, p);
-        if (kb > 0) tc_ld32(lane_addr + col, acc);
+        unsigned p[32];
+        tc_ld32(lane_addr + (unsigned)(pb * 128 + ch * 64 + cc * 32), p);
         tc_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-          const float v = __uint_as_float(p[i]) * s;
-          acc[i] = __float_as_uint(kb > 0 ? v + __uint_as_float(acc[i]) : v);
-        }
-        tc_st32(lane_addr + col, acc);
+        for (int i = 0; i < 32; ++i)
+          acc[h * 64 + cc * 32 + i] = fmaf(__uint_as_float(p[i]), s, acc[h * 64 + cc * 32 + i]);
       }
-      tc_wait_st();
       tc_fence_before();
-      mbar_arrive(&sc->pempty[h]);                // the partial buffer may be overwritten
+      mbar_arrive(&sc->pempty[pb]);               // the partial buffer may be overwritten
     }
     fx = nfx; f0 = nf0; f1 = nf1;
   }
   // the accumulator is complete
   if (g1) {
-    float o[64];
     float amax = 0.f;
 #pragma unroll
-    for (int cc = 0; cc < 2; ++cc) {
-      unsigned g[32], u[32];
-      tc_ld32(lane_addr + (unsigned)(ch * 64 + cc * 32), g);
-      tc_ld32(lane_addr + 128u + (unsigned)(ch * 64 + cc * 32), u);
-      tc_wait_ld();
-#pragma unroll
-      for (int i = 0; i < 32; ++i) {
-        const float gv = __uint_as_float(g[i]);
-        const float v = __fdividef(gv, 1.0f + __expf(-gv)) * __uint_as_float(u[i]);
-        o[cc * 32 + i] = v;
-        amax = fmaxf(amax, fabsf(v));
-      }
+    for (int i = 0; i < 64; ++i) {                // gate column i and up column i of this slice
+      const float gv = acc[i];
+      const float v = __fdividef(gv, 1.0f + __expf(-gv)) * acc[64 + i];
+      acc[i] = v;
+      amax = fmaxf(amax, fabsf(v));
     }
     // the row's 128 outputs live in two threads (ch = 0, 1): exchange the partial maxima
     sc->amax_x[ch][q][lane] = amax;
     mbar_arrive(&sc->xbar[q]);
-    if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->xbar[q], xph, 20))) return false;
+    if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->xbar[q], xph, 20))) return false;
     xph ^= 1u;
     amax = fmaxf(amax, sc->amax_x[ch ^ 1][q][lane]);
     const float scale = amax > 0.f ? amax / 448.0f : 1.0f;
@@ -402,37 +415,30 @@ __device__ inline bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev* op, cons
         unsigned w[4];
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
-          const float* v = o + j * 16 + i * 4;
-          const unsigned lo = __nv_cvt_float2_to_fp8x2(make_float2(v[0] * inv, v[1] * inv), __NV_SATFINITE, __NV_E4M3);
-          const unsigned hi = __nv_cvt_float2_to_fp8x2(make_float2(v[2] * inv, v[3] * inv), __NV_SATFINITE, __NV_E4M3);
+          const int b0 = j * 16 + i * 4;
+          const unsigned lo = __nv_cvt_float2_to_fp8x2(make_float2(acc[b0] * inv, acc[b0 + 1] * inv), __NV_SATFINITE, __NV_E4M3);
+          const unsigned hi = __nv_cvt_float2_to_fp8x2(make_float2(acc[b0 + 2] * inv, acc[b0 + 3] * inv), __NV_SATFINITE, __NV_E4M3);
           w[i] = lo | (hi << 16);
         }
         reinterpret_cast<uint4*>(dst)[j] = make_uint4(w[0], w[1], w[2], w[3]);
       }
       if (ch == 0) op->a_scale[(size_t)(ti.row0 + row) * IB + ti.n] = scale;
     }
-  } else {
+  } else if (valid) {
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
+      __nv_bfloat16* dst = op->D + (size_t)(ti.row0 + row) * a.H + (size_t)ti.n * kTileN2 + h * 128 + ch * 64;
 #pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        unsigned v[32];
-        tc_ld32(lane_addr + (unsigned)(h * 128 + ch * 64 + cc * 32), v);
-        tc_wait_ld();
-        if (valid) {
-          __nv_bfloat16* dst = op->D + (size_t)(ti.row0 + row) * a.H + (size_t)ti.n * kTileN2 + h * 128 + ch * 64 + cc * 32;
-          uint4 o4[4];
-          __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(o4);
+      for (int j = 0; j < 8; ++j) {
+        uint4 o4;
+        __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o4);
 #pragma unroll
-          for (int i = 0; i < 16; ++i)
-            oh[i] = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
-#pragma unroll
-          for (int i = 0; i < 4; ++i) reinterpret_cast<uint4*>(dst)[i] = o4[i];
-        }
+        for (int i = 0; i < 4; ++i)
+          oh[i] = __floats2bfloat162_rn(acc[h * 64 + j * 8 + 2 * i], acc[h * 64 + j * 8 + 2 * i + 1]);
+        reinterpret_cast<uint4*>(dst)[j] = o4;
       }
     }
   }
-  tc_fence_before();
   return true;
 }
 
@@ -465,10 +471,13 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       mbar_init(&sc->full[s], 1);
       mbar_init(&sc->fullA[s], kGatherThreads);
       mbar_init(&sc->empty[s], 1);
+      mbar_init(&sc->emptyA[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sc->tfull[s], 1);
       mbar_init(&sc->tempty[s], 256);
+    }
+    for (int s = 0; s < 4; ++s) {
       mbar_init(&sc->pfull[s], 1);
       mbar_init(&sc->pempty[s], 256);
     }
@@ -494,8 +503,14 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
   __syncthreads();
   tc_fence_after();
   const unsigned tmem = sc->tmem_base;
+  // The fp8 epilogue keeps 128 fp32 accumulators per thread: the two epilogue warpgroups take
+  // registers from the two others (56 + 200 = 2 x 128 per thread pair).  Each role changes its
+  // allowance at the top of its own branch, so the compiler can budget the branch by it.
+#define MOE_REGS_DEC() do { if constexpr (kFp8) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); } while (0)
+#define MOE_REGS_INC() do { if constexpr (kFp8) asm volatile("setmaxnreg.inc.sync.aligned.u32 200;"); } while (0)
 
   if (warp == 0) {
+    MOE_REGS_DEC();
     // ============================================================ scheduler + TMA producer
     // The next tile is claimed while the current one is still being loaded (after its
     // kClaimAt-th k-block), so the claim's round trips and the first loads of the next tile
@@ -559,6 +574,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #endif
             unsigned char* sA = stages + (size_t)stage * kStageBytes;
             unsigned char* sB = sA + kABytes;
+            if (g1) mbar_arrive(&sc->emptyA[stage]);      // the gather warps may fill this stage
             mbar_expect_tx(&sc->full[stage], tx);
             tma_tile_2d(sB, tmw, kb * kKb, wrow0, &sc->full[stage]);
             tma_tile_2d(sB + kBHalfBytes, tmw, kb * kKb, wrow1, &sc->full[stage]);
@@ -606,12 +622,13 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       }
     }
   } else if (warp == 1) {
+    MOE_REGS_DEC();
     // ============================================================ MMA issuer
 #ifdef MOE_TIMING_PROBE
     int dbg_i = 0;
 #endif
     int stage = 0, islot = 0;
-    unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0, pph[2] = {0, 0};
+    unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0, pph = 0;
     AccUse accs;
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 6))) break;
@@ -632,8 +649,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
             phA ^= 1u << stage;
           }
           for (int h = 0; h < 2 && !fail; ++h) {
-            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->pempty[h], pph[h] ^ 1u, 18))) { fail = true; break; }
-            pph[h] ^= 1u;
+            const int pb = h * 2 + (kb & 1);              // partial buffer of this half and k-block
+            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->pempty[pb], ((pph >> pb) & 1u) ^ 1u, 18))) { fail = true; break; }
+            pph ^= 1u << pb;
             tc_fence_after();
             if (lane == 0) {
               fence_async_proxy_smem();
@@ -642,8 +660,8 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
               const unsigned long long bd = umma_desc(sA + kABytes + h * kBHalfBytes, kRowBytes);
 #pragma unroll
               for (int k4 = 0; k4 < 4; ++k4)            // 32 e4m3 elements (32 bytes) per step
-                tc_mma_f8(tmem + kPartialCol + (unsigned)h * 128u, ad + 2ull * k4, bd + 2ull * k4, kIdescF8, k4 ? 1u : 0u);
-              tc_commit(&sc->pfull[h]);
+                tc_mma_f8(tmem + (unsigned)pb * 128u, ad + 2ull * k4, bd + 2ull * k4, kIdescF8, k4 ? 1u : 0u);
+              tc_commit(&sc->pfull[pb]);
               if (h == 1) tc_commit(&sc->empty[stage]);
             }
             __syncwarp();
@@ -707,6 +725,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
     }
   } else if (warp >= 4 && warp < 4 + kGatherThreads / 32) {
+    MOE_REGS_DEC();
     // ============================================================ gather warps (cp.async)
     // Rows of a gate/up tile are scattered tokens: row r of the tile is token
     // sorted_to_flat[row0 + r] / k.  Adjacent lanes copy one row slice (16 bytes each)
@@ -717,7 +736,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     constexpr int kPasses = 256 / kRowsPerPass;
     const int chunk = gt % kCpr, rbase = gt / kCpr;       // rows rbase + kRowsPerPass * j
     int islot = 0;
-    unsigned iph = 0, kiter = 0;                          // kiter: k-blocks of all GEMM tiles so far
+    unsigned iph = 0, kiter = 0, phE = 0;                 // kiter: k-blocks of all GEMM tiles so far
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 13))) break;
       const int kind = sc->info[islot].kind;
@@ -728,15 +747,8 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
       if (kind == kEnd) break;
       if (kind == kCombine) continue;
-      if (kind == kDown) {
-        // nothing to gather, but keep in step with the stage ring: a parity wait is only
-        // meaningful for a waiter that is at most one phase ahead of the barrier
-        bool failed = false;
-        for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
-          const int stage = (int)(kiter % kStages);
-          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kStages) & 1u) ^ 1u, 15))) { failed = true; break; }
-        }
-        if (failed) break;
+      if (kind == kDown) {             // nothing to gather; only the stage index moves on
+        kiter += (unsigned)kblocks;
         continue;
       }
       const OpDev* op = &args.ops[slot];
@@ -750,9 +762,12 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       }
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
+        // The producer relays "stage free" for gate/up k-blocks through emptyA: that barrier
+        // advances only when this warp takes part, so its parity never aliases (a parity wait is
+        // only meaningful for a waiter within one phase of the barrier).
         const int stage = (int)(kiter % kStages);
-        const unsigned ph = (kiter / kStages) & 1u;
-        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 14))) { fail = true; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->emptyA[stage], (phE >> stage) & 1u, 14))) { fail = true; break; }
+        phE ^= 1u << stage;
         const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
         const unsigned char* Xk = X + (size_t)kb * kRowBytes;
 #pragma unroll
@@ -769,6 +784,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     }
     cp_async_wait_all();
   } else if (warp == 2) {
+    MOE_REGS_DEC();
     // ============================================================ committer
     // Publishes a tile once all epilogue threads have arrived on the tile's barrier: the
     // barrier orders their stores before this warp's fence and release (cumulativity).
@@ -789,6 +805,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
     }
   } else if (warp >= 8) {
+    MOE_REGS_INC();
     // ============================================================ epilogue (8 warps)
     // Warp w may read TMEM lanes 32 (w % 4) .. +31, i.e. accumulator rows of that quadrant.
     // The two warps of a quadrant split the columns of every accumulator the tile used.
@@ -796,12 +813,12 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     const int half = (warp - 8) >> 2;             // which half of the columns
     const int etid = threadIdx.x - 256;           // 0..255
     int islot = 0;
-    unsigned iph = 0, aph[2] = {0, 0}, eph[2] = {0, 0}, xph = 0;
+    unsigned iph = 0, aph[2] = {0, 0}, eph = 0, xph = 0;
     AccUse accs;
     unsigned char* scratch = sc->epi_scratch[warp - 8];
     const int srow = lane >> 2, schunk = lane & 3;          // this lane's part of a store
     while (true) {
-      if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 9))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->ifull[islot], iph, 9))) break;
       const TileInfo ti = sc->info[islot];
       if (ti.kind == kEnd) break;
       OpDev* op = &args.ops[ti.slot];
@@ -820,7 +837,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
           if (!use[b]) continue;
-          ok = __all_sync(0xffffffffu, mbar_wait(c, &sc->tfull[b], aph[b], 10));
+          ok = __all_sync(0xffffffffu, mbar_wait_inline(c, &sc->tfull[b], aph[b], 10));
           if (!ok) break;
           aph[b] ^= 1u;
           tc_fence_after();
@@ -881,6 +898,10 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       mbar_arrive(&sc->done[islot]);              // this thread's part of the tile is stored
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
     }
+  }
+
+  else {
+    MOE_REGS_DEC();        // warp 3: idle, but its warpgroup changes its allowance together
   }
 
   // teardown: nothing is claimed any more; let asynchronous work settle, then free TMEM
