@@ -261,7 +261,7 @@ class Context:
         self.workspace_bytes = nbytes
 
     def close(self):
-        if getattr(self, "ctx", None):
+        if getattr(self, "ctx", None) and moe_destroy is not None:    # None at interpreter shutdown
             moe_destroy(self.ctx)
             self.ctx = None
 

@@ -85,7 +85,8 @@ struct __align__(128) OpDev {
   __nv_bfloat16* D;      // [Rmax, H]  expert output, packed order
   MTile* mtiles;         // [max_mtiles]
   int4* tile_list;       // [max_tiles] queue entries in claim order
-  int* plan_hist;        // [n_chunks, E] per-warp histogram, then per-warp base rank
+  int* plan_hist;        // [n_chunks, E] per-warp histogram
+  int* plan_base;        // [n_chunks, E] per-warp base rank of each expert
   PlanState* plan;
   RunState* run;
   int* g1_done;          // [max_mtiles] committed gate/up tiles per work tile

@@ -61,7 +61,7 @@ Layout make_layout(const moe_config_t* c) {
   L.D_off = off;       off = align_up(off + (size_t)L.max_rows * H * 2, 1024);
   L.mtiles_off = off;  off = align_up(off + (size_t)L.max_mtiles * sizeof(MTile), 1024);
   L.tiles_off = off;   off = align_up(off + (size_t)L.max_tiles * sizeof(int4), 1024);
-  L.hist_off = off;    off = align_up(off + n_chunks * E * 4, 1024);
+  L.hist_off = off;    off = align_up(off + 2 * n_chunks * E * 4, 1024);   // histogram + base ranks
   L.plan_off = off;    off = align_up(off + sizeof(PlanState), 1024);
   L.slot_stride = off;
 
@@ -93,6 +93,8 @@ struct moe_ctx {
   EncodeTiledFn encode;
   moe_op_t ops[kMaxOps];
   bool planned[kMaxOps];
+  OpDev host_ops[kMaxOps];      // what the device copy of each slot holds (tensor maps included)
+  bool uploaded[kMaxOps];
   Global* g() const { return reinterpret_cast<Global*>(ws + L.global_off); }
   RunHead* rh() const { return reinterpret_cast<RunHead*>(ws + L.runzero_off); }
   unsigned char* slot_base(int s) const { return ws + L.slots_off + L.slot_stride * s; }
@@ -123,6 +125,14 @@ int make_map(moe_ctx* ctx, CUtensorMap* out, const void* base, size_t rows, size
 
 // a stream-ordered 4-byte write: the value travels in the launch, not through host memory
 __global__ void set_word_kernel(int* p, int v) { *reinterpret_cast<volatile int*>(p) = v; }
+
+// The op descriptor travels as a kernel parameter (no pageable-memory copy on the stream).
+__global__ void write_op_kernel(const __grid_constant__ OpDev src, OpDev* dst) {
+  const int n = (int)(sizeof(OpDev) / sizeof(int));
+  const int* s = reinterpret_cast<const int*>(&src);
+  int* d = reinterpret_cast<int*>(dst);
+  for (int i = threadIdx.x; i < n; i += blockDim.x) d[i] = s[i];
+}
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15) == 0; }
 
@@ -178,6 +188,7 @@ int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_c
   ctx->n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : sms;
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   memset(ctx->planned, 0, sizeof(ctx->planned));
+  memset(ctx->uploaded, 0, sizeof(ctx->uploaded));
   // zero the control blocks (status, budget, run state, plan states)
   cudaError_t e = cudaMemset(ctx->ws, 0, L.slots_off);
   for (int s = 0; s < cfg->max_ops && e == cudaSuccess; ++s)
@@ -227,22 +238,30 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   h.mtiles = reinterpret_cast<MTile*>(sb + L.mtiles_off);
   h.tile_list = reinterpret_cast<int4*>(sb + L.tiles_off);
   h.plan_hist = reinterpret_cast<int*>(sb + L.hist_off);
+  h.plan_base = h.plan_hist + (((size_t)L.max_rows + kPlanChunk - 1) / kPlanChunk) * c.n_experts;
   h.plan = reinterpret_cast<PlanState*>(sb + L.plan_off);
   h.run = reinterpret_cast<RunState*>(ctx->rs_base(slot));
   h.g1_done = reinterpret_cast<int*>(ctx->rs_base(slot) + sizeof(RunState));
-  int rc = MOE_OK;
-  if (op->n_tokens > 0) {
-    rc = make_map(ctx, &h.tm_a8, h.A, (size_t)L.max_rows, (size_t)c.inter, 8);
-    if (!rc) rc = make_map(ctx, &h.tm_a32, h.A, (size_t)L.max_rows, (size_t)c.inter, 32);
-    if (!rc) rc = make_map(ctx, &h.tm_a128, h.A, (size_t)L.max_rows, (size_t)c.inter, 128);
-    if (!rc) rc = make_map(ctx, &h.tm_a256, h.A, (size_t)L.max_rows, (size_t)c.inter, 256);
-    if (!rc) rc = make_map(ctx, &h.tm_w1, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 128);
-    if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
-    if (rc) return rc;
-  }
+  // Re-planning a slot with the same buffers (the usual serving loop) reuses the descriptors
+  // already on the device: encoding seven tensor maps and uploading them is host time.
+  const bool same = ctx->uploaded[slot] && memcmp(&ctx->ops[slot], op, sizeof(moe_op_t)) == 0;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(ctx->op_dev(slot), &h, sizeof(h), cudaMemcpyHostToDevice, st) != cudaSuccess)
-    return MOE_ECUDA;
+  if (!same) {
+    int rc = MOE_OK;
+    if (op->n_tokens > 0) {
+      rc = make_map(ctx, &h.tm_a8, h.A, (size_t)L.max_rows, (size_t)c.inter, 8);
+      if (!rc) rc = make_map(ctx, &h.tm_a32, h.A, (size_t)L.max_rows, (size_t)c.inter, 32);
+      if (!rc) rc = make_map(ctx, &h.tm_a128, h.A, (size_t)L.max_rows, (size_t)c.inter, 128);
+      if (!rc) rc = make_map(ctx, &h.tm_a256, h.A, (size_t)L.max_rows, (size_t)c.inter, 256);
+      if (!rc) rc = make_map(ctx, &h.tm_w1, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 128);
+      if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
+      if (rc) return rc;
+    }
+    write_op_kernel<<<1, 128, 0, st>>>(h, ctx->op_dev(slot));
+    if (cudaGetLastError() != cudaSuccess) return MOE_ECUDA;
+    ctx->host_ops[slot] = h;
+    ctx->uploaded[slot] = true;
+  }
   if (launch_plan(ctx->op_dev(slot), ctx->g(), slot, op->n_tokens, c.top_k, c.n_experts, L.NT1, L.NT2,
                   c.dtype == MOE_DTYPE_FP8_E4M3 ? kWorkRowsFp8 : kWorkRowsBf16, st) != cudaSuccess)
     return MOE_ECUDA;

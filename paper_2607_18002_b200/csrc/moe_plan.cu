@@ -25,15 +25,19 @@ plan_hist_kernel(const OpDev* __restrict__ op, Global* g, int slot, int R, int E
   __syncwarp();
   const int* ids = op->topk_ids;
   const int base = chunk * kPlanChunk;
+  int my[kPlanChunk / 32];                    // this lane's ids of the chunk, loaded up front
+#pragma unroll
   for (int it = 0; it < kPlanChunk / 32; ++it) {
     const int i = base + it * 32 + lane;
-    int id = -1;
-    if (i < R) {
-      id = ids[i];
-      if (id < 0 || id >= E) {
-        report(&g->status, MOE_EBADID, slot, i, id, 0);
-        id = -1;
-      }
+    my[it] = i < R ? ids[i] : -1;
+  }
+#pragma unroll
+  for (int it = 0; it < kPlanChunk / 32; ++it) {
+    const int i = base + it * 32 + lane;
+    int id = my[it];
+    if (i < R && (id < 0 || id >= E)) {
+      report(&g->status, MOE_EBADID, slot, i, id, 0);
+      id = -1;
     }
     const unsigned peers = __match_any_sync(0xffffffffu, id);
     if (id >= 0 && (peers & ((1u << lane) - 1)) == 0) h[id] += __popc(peers);
@@ -78,31 +82,52 @@ __global__ void __launch_bounds__(1024)
 plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int NT1, int NT2,
                  int T, int work_rows) {
   __shared__ int warp_sums[33];
-  __shared__ int s_cnt[kMaxExperts], s_m0[kMaxExperts], s_grp[kMaxExperts], s_moff[kMaxExperts];
+  __shared__ int s_cnt[kMaxExperts], s_grp[kMaxExperts], s_moff[kMaxExperts], s_off[kMaxExperts];
+  __shared__ int s_part[1024];
   __shared__ int g_cnt[kMaxExperts], g_base1[kMaxExperts], g_base2[kMaxExperts];
   __shared__ int s_ntiles;
   const int e = threadIdx.x;
 
-  // column scan over the per-warp histograms: base rank of every (warp chunk, expert)
-  int cnt = 0;
-  if (e < E) {
-    int* hcol = op->plan_hist + e;
-    for (int c = 0; c < n_chunks; ++c) {
-      const int v = hcol[(size_t)c * E];
-      hcol[(size_t)c * E] = cnt;
-      cnt += v;
-    }
+  // column sums of the per-warp histograms, the device prefix sum over experts, then the base
+  // rank of every (warp chunk, expert).  Reads and writes use different arrays so that the
+  // loads of a column do not wait on the stores.
+  const int* __restrict__ hist = op->plan_hist;
+  int* __restrict__ base = op->plan_base;
+  // the 1024 threads split every expert's column into `parts` chunk ranges
+  const int parts = max(1, 1024 / E);
+  const int part = threadIdx.x / E, pe = threadIdx.x % E;
+  const int cpp = (n_chunks + parts - 1) / parts;
+  const int c0 = min(n_chunks, part * cpp), c1 = min(n_chunks, c0 + cpp);
+  int psum = 0;
+  if (part < parts) {
+#pragma unroll 8
+    for (int c = c0; c < c1; ++c) psum += hist[(size_t)c * E + pe];
+    s_part[part * E + pe] = psum;
   }
+  __syncthreads();
+  int cnt = 0;
+  if (e < E)
+    for (int p = 0; p < parts; ++p) cnt += s_part[p * E + e];
   int total;
   const int off = block_excl_scan(cnt, &total, warp_sums);       // device prefix sum over experts
   if (e < E) {
     op->counts[e] = cnt;
     op->offsets[e] = off;
-    int* hcol = op->plan_hist + e;
-    for (int c = 0; c < n_chunks; ++c) hcol[(size_t)c * E] += off;
     s_cnt[e] = cnt;
+    s_off[e] = off;
   }
   if (e == 0) op->offsets[E] = total;
+  __syncthreads();
+  if (part < parts) {
+    int run = s_off[pe];
+    for (int p = 0; p < part; ++p) run += s_part[p * E + pe];
+#pragma unroll 8
+    for (int c = c0; c < c1; ++c) {
+      const int v = hist[(size_t)c * E + pe];
+      base[(size_t)c * E + pe] = run;
+      run += v;
+    }
+  }
 
   // m-tiles: ceil(m_e / M_t) per expert with rows (the footprint x_moe)
   const int me = (e < E) ? (cnt + kTileM - 1) / kTileM : 0;
@@ -129,7 +154,6 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   const int we = (e < E) ? (cnt + work_rows - 1) / work_rows : 0;
   int n_work;
   const int w0 = block_excl_scan(we, &n_work, warp_sums);
-  if (e < E) s_m0[e] = w0;
   __syncthreads();
   if (threadIdx.x == 0) {
     int ng = 0, acc = 0;
@@ -187,19 +211,23 @@ plan_scatter_kernel(const OpDev* __restrict__ op, int R, int E) {
   const int base = chunk * kPlanChunk;
   if (base >= R) return;
   int* run = sm + warp * E;
-  const int* src = op->plan_hist + (size_t)chunk * E;
+  const int* src = op->plan_base + (size_t)chunk * E;
   for (int e = lane; e < E; e += 32) run[e] = src[e];
   __syncwarp();
   const int* ids = op->topk_ids;
   int* s2f = op->sorted_to_flat;
   int* f2s = op->flat_to_sorted;
+  int my[kPlanChunk / 32];
+#pragma unroll
   for (int it = 0; it < kPlanChunk / 32; ++it) {
     const int i = base + it * 32 + lane;
-    int id = -1;
-    if (i < R) {
-      id = ids[i];
-      if (id < 0 || id >= E) id = -1;       // reported by the histogram kernel
-    }
+    my[it] = i < R ? ids[i] : -1;
+  }
+#pragma unroll
+  for (int it = 0; it < kPlanChunk / 32; ++it) {
+    const int i = base + it * 32 + lane;
+    int id = my[it];
+    if (id < 0 || id >= E) id = -1;         // reported by the histogram kernel
     const unsigned peers = __match_any_sync(0xffffffffu, id);
     const unsigned before = peers & ((1u << lane) - 1);
     int p = -1;

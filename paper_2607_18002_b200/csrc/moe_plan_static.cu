@@ -27,7 +27,8 @@ namespace moe {
 
 constexpr int kStaticMaxRows = MOE_PLAN_STATIC_MAX_ROWS;
 constexpr int kStaticMaxExperts = MOE_PLAN_STATIC_MAX_EXPERTS;
-constexpr int kStaticChunks = kStaticMaxRows / kPlanChunk;
+constexpr int kStaticChunkRows = 256;                    // routed rows ranked by one warp
+constexpr int kStaticChunks = kStaticMaxRows / kStaticChunkRows;
 constexpr int kStaticThreads = 256;
 constexpr int kStaticWarps = kStaticThreads / 32;
 
@@ -39,11 +40,11 @@ static_hist_kernel(const int* __restrict__ ids, int* __restrict__ hist, int R, i
   __shared__ int sm[kStaticWarps * kStaticMaxExperts];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x * kStaticWarps + warp;
-  const int base = chunk * kPlanChunk;
+  const int base = chunk * kStaticChunkRows;
   int* h = sm + warp * E;
   for (int e = lane; e < E; e += 32) h[e] = 0;
   __syncwarp();
-  for (int it = 0; it < kPlanChunk / 32; ++it) {
+  for (int it = 0; it < kStaticChunkRows / 32; ++it) {
     const int i = base + it * 32 + lane;
     int id = -1;
     if (i < R) {
@@ -97,12 +98,12 @@ static_scatter_kernel(const int* __restrict__ ids, const int* __restrict__ hist,
   __shared__ int sm[kStaticWarps * kStaticMaxExperts];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int chunk = blockIdx.x * kStaticWarps + warp;
-  const int base = chunk * kPlanChunk;
+  const int base = chunk * kStaticChunkRows;
   if (base >= R) return;
   int* run = sm + warp * E;
   for (int e = lane; e < E; e += 32) run[e] = hist[(size_t)chunk * E + e];
   __syncwarp();
-  for (int it = 0; it < kPlanChunk / 32; ++it) {
+  for (int it = 0; it < kStaticChunkRows / 32; ++it) {
     const int i = base + it * 32 + lane;
     int id = -1;
     if (i < R) {
@@ -157,7 +158,7 @@ extern "C" int moe_plan_static(const int32_t* topk_ids, int32_t n_tokens, int32_
   const int rc = scratch_on_current_device(&scratch);
   if (rc != MOE_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  const int n_chunks = (R + kPlanChunk - 1) / kPlanChunk;
+  const int n_chunks = (R + kStaticChunkRows - 1) / kStaticChunkRows;
   const int blocks = (n_chunks + kStaticWarps - 1) / kStaticWarps;
   if (blocks > 0) static_hist_kernel<<<blocks, kStaticThreads, 0, st>>>(topk_ids, scratch, R, n_experts);
   static_scan_kernel<<<1, kStaticMaxExperts, 0, st>>>(scratch, n_chunks, n_experts, counts, offsets);
