@@ -376,13 +376,13 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
       tc_fence_after();
       const float s = fx * (h ? f1 : f0);
 #pragma unroll
-      for (int cc = 0; cc < 2; ++cc) {
-        unsigned p[32];
-        tc_ld32(lane_addr + (unsigned)(pb * 128 + ch * 64 + cc * 32), p);
+      for (int cc = 0; cc < 4; ++cc) {
+        unsigned p[16];
+        tc_ld16(lane_addr + (unsigned)(pb * 128 + ch * 64 + cc * 16), p);
         tc_wait_ld();
 #pragma unroll
-        for (int i = 0; i < 32; ++i)
-          acc[h * 64 + cc * 32 + i] = fmaf(__uint_as_float(p[i]), s, acc[h * 64 + cc * 32 + i]);
+        for (int i = 0; i < 16; ++i)
+          acc[h * 64 + cc * 16 + i] = fmaf(__uint_as_float(p[i]), s, acc[h * 64 + cc * 16 + i]);
       }
       tc_fence_before();
       mbar_arrive(&sc->pempty[pb]);               // the partial buffer may be overwritten
@@ -625,7 +625,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     MOE_REGS_DEC();
     // ============================================================ MMA issuer
 #ifdef MOE_TIMING_PROBE
-    int dbg_i = 0;
+    int dbg_i = 0, dbg_t = 0;
 #endif
     int stage = 0, islot = 0;
     unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0, pph = 0;
@@ -637,6 +637,10 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       const int rows = sc->info[islot].rows;
       if (kind == kEnd) break;
       bool fail = false;
+#ifdef MOE_TIMING_PROBE
+      const long long tt0 = clock64();
+      long long tt1 = 0, tt2 = 0;
+#endif
       if (kFp8 && kind != kCombine) {
         // FP8 with fp32 block scales: the tensor core cannot apply a scale per 128-deep K block,
         // so every k-block (= one scale block) is multiplied into a FRESH partial buffer, one
@@ -673,10 +677,15 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       } else if (kind != kCombine) {
         bool use0, use1;
         accs.take(rows, use0, use1);
-        if (use0 && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[0], aph[0] ^ 1u, 7))) break;
-        if (use1 && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[1], aph[1] ^ 1u, 7))) break;
-        tc_fence_after();
+        // A 256-row tile takes both accumulators: it waits for accumulator 1 only when its first
+        // MMA into it is due, so the drain of accumulator 1 overlaps the tile's first MMAs.
         const bool pair = use0 && use1;
+        if (use0 && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[0], aph[0] ^ 1u, 7))) break;
+        if (use1 && !pair && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[1], aph[1] ^ 1u, 7))) break;
+        tc_fence_after();
+#ifdef MOE_TIMING_PROBE
+        tt1 = clock64();
+#endif
         const unsigned d0 = tmem + (use0 ? 0u : (unsigned)kAccCols);     // accumulator of rows 0..127
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
@@ -698,6 +707,17 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #pragma unroll
             for (int k4 = 0; k4 < kBlockK / 16; ++k4)   // +32 bytes along K per step (>>4 = 2)
               tc_mma_bf16(d0, ad + 2ull * k4, bd + 2ull * k4, kIdesc, (kb | k4) ? 1u : 0u);
+          }
+          if (pair && kb == 0) {                         // accumulator 1 is needed from here on
+            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[1], aph[1] ^ 1u, 7))) { fail = true; break; }
+            tc_fence_after();
+#ifdef MOE_TIMING_PROBE
+            tt2 = clock64();
+#endif
+          }
+          if (lane == 0) {
+            const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
+            const unsigned long long bd = umma_desc(sA + kABytes, kRowBytes);
             if (pair) {                                  // rows 128..255 against the same weight tile
               const unsigned long long ad1 = umma_desc(sA + kAHalfBytes, kRowBytes);
 #pragma unroll
@@ -716,6 +736,12 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         if (lane == 0) {                                 // accumulator(s) complete
           if (use0) tc_commit(&sc->tfull[0]);
           if (use1) tc_commit(&sc->tfull[1]);
+#ifdef MOE_TIMING_PROBE
+          if (blockIdx.x == 7 && dbg_t < 512) {
+            long long* pp = args.dbg + 8192 * 4 + (size_t)dbg_t++ * 8;
+            pp[0] = tt0; pp[1] = tt1; pp[2] = tt2; pp[3] = clock64(); pp[4] = kind * 1000 + rows;
+          }
+#endif
         }
         __syncwarp();
         if (use0) aph[0] ^= 1u;
@@ -815,6 +841,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     int islot = 0;
     unsigned iph = 0, aph[2] = {0, 0}, eph = 0, xph = 0;
     AccUse accs;
+#ifdef MOE_TIMING_PROBE
+    int dbg_e = 0;
+#endif
     unsigned char* scratch = sc->epi_scratch[warp - 8];
     const int srow = lane >> 2, schunk = lane & 3;          // this lane's part of a store
     while (true) {
@@ -837,10 +866,16 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
           if (!use[b]) continue;
+#ifdef MOE_TIMING_PROBE
+          const long long te0 = clock64();
+#endif
           ok = __all_sync(0xffffffffu, mbar_wait_inline(c, &sc->tfull[b], aph[b], 10));
           if (!ok) break;
           aph[b] ^= 1u;
           tc_fence_after();
+#ifdef MOE_TIMING_PROBE
+          const long long te1 = clock64();
+#endif
           const int rbase = pair ? b * kTileM : 0;               // first tile row of this accumulator
           const int nrows = min(ti.rows - rbase, kTileM);
           if (q * 32 < nrows) {
@@ -852,16 +887,18 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
                                  (size_t)(ti.row0 + rbase + q * 32) * pitch +
                                  (size_t)ti.n * (g1 ? kTileN1 : kTileN2) * 2;
             const int rows_here = min(32, nrows - q * 32);
+            // The TMEM load of pass p+1 is issued as soon as pass p has been converted, so its
+            // latency hides behind the transpose and the stores of pass p.
+            unsigned g[32], u[32];
+            tc_ld32(taddr + (half * passes) * 32 + (g1 ? 0 : 0), g);
+            if (g1) tc_ld32(taddr + 128 + (half * passes) * 32, u);
 #pragma unroll 1
             for (int p = 0; p < passes; ++p) {
               const int pass = half * passes + p;
               uint4 o[4];
               __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(o);
+              tc_wait_ld();
               if (g1) {
-                unsigned g[32], u[32];
-                tc_ld32(taddr + pass * 32, g);
-                tc_ld32(taddr + 128 + pass * 32, u);
-                tc_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i) {
                   const float a0 = silu_mul(__uint_as_float(g[2 * i]), __uint_as_float(u[2 * i]));
@@ -869,12 +906,13 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
                   oh[i] = __floats2bfloat162_rn(a0, a1);
                 }
               } else {
-                unsigned v[32];
-                tc_ld32(taddr + pass * 32, v);
-                tc_wait_ld();
 #pragma unroll
                 for (int i = 0; i < 16; ++i)
-                  oh[i] = __floats2bfloat162_rn(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1]));
+                  oh[i] = __floats2bfloat162_rn(__uint_as_float(g[2 * i]), __uint_as_float(g[2 * i + 1]));
+              }
+              if (p + 1 < passes) {
+                tc_ld32(taddr + (pass + 1) * 32, g);
+                if (g1) tc_ld32(taddr + 128 + (pass + 1) * 32, u);
               }
               __syncwarp();                                          // scratch free again
 #pragma unroll
@@ -892,6 +930,12 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           }
           tc_fence_before();
           mbar_arrive(&sc->tempty[b]);            // accumulator may be overwritten
+#ifdef MOE_TIMING_PROBE
+          if (blockIdx.x == 7 && warp == 8 && lane == 0 && dbg_e < 1024) {
+            long long* pp = args.dbg + 12288 * 4 + (size_t)dbg_e++ * 4;
+            pp[0] = te0; pp[1] = te1; pp[2] = clock64(); pp[3] = ti.kind * 1000 + ti.rows + b * 100000;
+          }
+#endif
         }
       }
       if (!ok) break;
