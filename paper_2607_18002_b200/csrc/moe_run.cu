@@ -52,9 +52,9 @@ struct TileInfo {
 };
 
 struct SharedCtl {
-  unsigned long long full[kStages], fullA[kStages], empty[kStages], emptyA[kStages];
+  unsigned long long full[kStages], fullA[kStages], empty[kStages];
   unsigned long long tfull[2], tempty[2];
-  unsigned long long pfull[4], pempty[4];          // fp8: per-k-block partial products: [column half][2 buffers]
+  unsigned long long pfull[2], pempty[2];          // fp8: per-k-block partial products, two 256-column buffers
   unsigned long long xbar[4];                      // fp8: amax exchange between the two warps of a quadrant
   float amax_x[2][4][32];
   unsigned long long ifull[kRing], iempty[kRing], done[kRing];
@@ -328,8 +328,8 @@ __device__ __forceinline__ float silu_mul(float g, float u) {
 }
 
 // ------------------------------------------------------------------ FP8 (e4m3, fp32 block scales)
-// instruction descriptor: D fp32, A/B e4m3, both K-major, M = 128, N = 128
-constexpr unsigned kIdescF8 = (1u << 4) | ((128u >> 3) << 17) | ((128u >> 4) << 24);
+// instruction descriptor: D fp32, A/B e4m3, both K-major, M = 128, N = 256
+constexpr unsigned kIdescF8 = (1u << 4) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
 
 // One e4m3 tile on the epilogue warps.  Thread = (accumulator row, 64-column slice of each
 // 128-column half); its 128 fp32 accumulators stay in registers (the epilogue warps raise
@@ -363,31 +363,51 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
   float acc[128];                                 // [half][64]
 #pragma unroll
   for (int i = 0; i < 128; ++i) acc[i] = 0.f;
-  float fx = sx[0], f0 = sw0[0], f1 = sw1[0];
+  float4 vx = make_float4(0.f, 0.f, 0.f, 0.f), v0 = vx, v1 = vx;   // scales of four k-blocks at a time
   for (int kb = 0; kb < ti.kblocks; ++kb) {
-    float nfx = 0.f, nf0 = 0.f, nf1 = 0.f;
-    if (kb + 1 < ti.kblocks) { nfx = sx[kb + 1]; nf0 = sw0[kb + 1]; nf1 = sw1[kb + 1]; }
+    if ((kb & 3) == 0) {
+      // the scale rows are contiguous over k-blocks; their lengths (H/128, I/128) are multiples of 4
+      // for the supported shapes, else fall back to scalar loads
+      if (((ti.kblocks & 3) == 0)) {
+        vx = *reinterpret_cast<const float4*>(sx + kb);
+        v0 = *reinterpret_cast<const float4*>(sw0 + kb);
+        v1 = *reinterpret_cast<const float4*>(sw1 + kb);
+      } else {
+        float tx[4], t0[4], t1[4];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-      const int pb = h * 2 + (kb & 1);
-      if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->pfull[pb], (eph >> pb) & 1u, 19))) return false;
-      eph ^= 1u << pb;
-
-      tc_fence_after();
-      const float s = fx * (h ? f1 : f0);
-#pragma unroll
-      for (int cc = 0; cc < 4; ++cc) {
-        unsigned p[16];
-        tc_ld16(lane_addr + (unsigned)(pb * 128 + ch * 64 + cc * 16), p);
-        tc_wait_ld();
-#pragma unroll
-        for (int i = 0; i < 16; ++i)
-          acc[h * 64 + cc * 16 + i] = fmaf(__uint_as_float(p[i]), s, acc[h * 64 + cc * 16 + i]);
+        for (int i = 0; i < 4; ++i) {
+          const int kk = min(kb + i, ti.kblocks - 1);
+          tx[i] = sx[kk]; t0[i] = sw0[kk]; t1[i] = sw1[kk];
+        }
+        vx = make_float4(tx[0], tx[1], tx[2], tx[3]);
+        v0 = make_float4(t0[0], t0[1], t0[2], t0[3]);
+        v1 = make_float4(t1[0], t1[1], t1[2], t1[3]);
       }
-      tc_fence_before();
-      mbar_arrive(&sc->pempty[pb]);               // the partial buffer may be overwritten
     }
-    fx = nfx; f0 = nf0; f1 = nf1;
+    const int sub = kb & 3;
+    const float fx = sub == 0 ? vx.x : (sub == 1 ? vx.y : (sub == 2 ? vx.z : vx.w));
+    const float s0 = fx * (sub == 0 ? v0.x : (sub == 1 ? v0.y : (sub == 2 ? v0.z : v0.w)));
+    const float s1 = fx * (sub == 0 ? v1.x : (sub == 1 ? v1.y : (sub == 2 ? v1.z : v1.w)));
+    const int pb = kb & 1;
+    if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->pfull[pb], (eph >> pb) & 1u, 19))) return false;
+    eph ^= 1u << pb;
+    tc_fence_after();
+    // eight 16-column chunks (four per half); the load of chunk c+1 is in flight while chunk c
+    // is multiplied in
+    const unsigned pbase = lane_addr + (unsigned)(pb * 256 + ch * 64);
+    unsigned p[2][16];
+    tc_ld16(pbase, p[0]);
+#pragma unroll
+    for (int cc = 0; cc < 8; ++cc) {
+      tc_wait_ld();
+      if (cc + 1 < 8) tc_ld16(pbase + (unsigned)(((cc + 1) >> 2) * 128 + ((cc + 1) & 3) * 16), p[(cc + 1) & 1]);
+      const float s = (cc >> 2) ? s1 : s0;
+#pragma unroll
+      for (int i = 0; i < 16; ++i)
+        acc[cc * 16 + i] = fmaf(__uint_as_float(p[cc & 1][i]), s, acc[cc * 16 + i]);
+    }
+    tc_fence_before();
+    mbar_arrive(&sc->pempty[pb]);                 // the partial buffer may be overwritten
   }
   // the accumulator is complete
   if (g1) {
@@ -471,13 +491,12 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       mbar_init(&sc->full[s], 1);
       mbar_init(&sc->fullA[s], kGatherThreads);
       mbar_init(&sc->empty[s], 1);
-      mbar_init(&sc->emptyA[s], 1);
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sc->tfull[s], 1);
       mbar_init(&sc->tempty[s], 256);
     }
-    for (int s = 0; s < 4; ++s) {
+    for (int s = 0; s < 2; ++s) {
       mbar_init(&sc->pfull[s], 1);
       mbar_init(&sc->pempty[s], 256);
     }
@@ -504,10 +523,10 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
   tc_fence_after();
   const unsigned tmem = sc->tmem_base;
   // The fp8 epilogue keeps 128 fp32 accumulators per thread: the two epilogue warpgroups take
-  // registers from the two others (56 + 200 = 2 x 128 per thread pair).  Each role changes its
+  // registers from the two others (64 + 192 = 2 x 128 per thread pair).  Each role changes its
   // allowance at the top of its own branch, so the compiler can budget the branch by it.
-#define MOE_REGS_DEC() do { if constexpr (kFp8) asm volatile("setmaxnreg.dec.sync.aligned.u32 56;"); } while (0)
-#define MOE_REGS_INC() do { if constexpr (kFp8) asm volatile("setmaxnreg.inc.sync.aligned.u32 200;"); } while (0)
+#define MOE_REGS_DEC() do { if constexpr (kFp8) asm volatile("setmaxnreg.dec.sync.aligned.u32 64;"); } while (0)
+#define MOE_REGS_INC() do { if constexpr (kFp8) asm volatile("setmaxnreg.inc.sync.aligned.u32 192;"); } while (0)
 
   if (warp == 0) {
     MOE_REGS_DEC();
@@ -574,7 +593,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #endif
             unsigned char* sA = stages + (size_t)stage * kStageBytes;
             unsigned char* sB = sA + kABytes;
-            if (g1) mbar_arrive(&sc->emptyA[stage]);      // the gather warps may fill this stage
             mbar_expect_tx(&sc->full[stage], tx);
             tma_tile_2d(sB, tmw, kb * kKb, wrow0, &sc->full[stage]);
             tma_tile_2d(sB + kBHalfBytes, tmw, kb * kKb, wrow1, &sc->full[stage]);
@@ -647,26 +665,38 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         // per 128-column half of the weight tile (each half has a single weight scale), and the
         // epilogue warps scale-and-add it into the fp32 accumulator columns of TMEM.
         for (int kb = 0; kb < kblocks; ++kb) {
+#ifdef MOE_TIMING_PROBE
+          const long long q0 = clock64();
+#endif
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
-          if (kind == kGateUp) {
-            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], (phA >> stage) & 1u, 12))) { fail = true; break; }
-            phA ^= 1u << stage;
-          }
-          for (int h = 0; h < 2 && !fail; ++h) {
-            const int pb = h * 2 + (kb & 1);              // partial buffer of this half and k-block
+#ifdef MOE_TIMING_PROBE
+          const long long q1 = clock64();
+#endif
+          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], ph, 12))) { fail = true; break; }
+#ifdef MOE_TIMING_PROBE
+          const long long q2 = clock64();
+#endif
+          {
+            const int pb = kb & 1;                        // partial buffer of this k-block
             if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->pempty[pb], ((pph >> pb) & 1u) ^ 1u, 18))) { fail = true; break; }
             pph ^= 1u << pb;
             tc_fence_after();
+#ifdef MOE_TIMING_PROBE
+            if (blockIdx.x == 7 && lane == 0 && dbg_i < 4096) {
+              long long* pp = args.dbg + (size_t)dbg_i++ * 4;
+              pp[0] = q0; pp[1] = q1; pp[2] = q2; pp[3] = clock64();
+            }
+#endif
             if (lane == 0) {
               fence_async_proxy_smem();
               const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
               const unsigned long long ad = umma_desc(sA, kRowBytes);
-              const unsigned long long bd = umma_desc(sA + kABytes + h * kBHalfBytes, kRowBytes);
+              const unsigned long long bd = umma_desc(sA + kABytes, kRowBytes);
 #pragma unroll
-              for (int k4 = 0; k4 < 4; ++k4)            // 32 e4m3 elements (32 bytes) per step
-                tc_mma_f8(tmem + (unsigned)pb * 128u, ad + 2ull * k4, bd + 2ull * k4, kIdescF8, k4 ? 1u : 0u);
+              for (int k4 = 0; k4 < 4; ++k4)              // 32 e4m3 elements (32 bytes) per step
+                tc_mma_f8(tmem + (unsigned)(pb * 256), ad + 2ull * k4, bd + 2ull * k4, kIdescF8, k4 ? 1u : 0u);
               tc_commit(&sc->pfull[pb]);
-              if (h == 1) tc_commit(&sc->empty[stage]);
+              tc_commit(&sc->empty[stage]);
             }
             __syncwarp();
           }
@@ -692,10 +722,10 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #ifdef MOE_TIMING_PROBE
           const long long t_fullB = clock64();
 #endif
-          if (kind == kGateUp) {       // gathered rows arrive through their own barrier
-            if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], (phA >> stage) & 1u, 12))) { fail = true; break; }
-            phA ^= 1u << stage;
-          }
+          // The gather warps arrive on fullA for every k-block (with the copied rows of a
+          // gate/up tile, empty-handed otherwise): being part of every stage hand-off keeps them
+          // within one phase of the stage barriers they wait on.
+          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], ph, 12))) { fail = true; break; }
           tc_fence_after();
           if (lane == 0) {
 #ifdef MOE_TIMING_PROBE
@@ -759,10 +789,10 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     const int gt = threadIdx.x - 128;
     constexpr int kCpr = kRowBytes / 16;                  // 16-byte chunks per row slice
     constexpr int kRowsPerPass = kGatherThreads / kCpr;   // rows covered by one cp.async per thread
-    constexpr int kPasses = 256 / kRowsPerPass;
+    constexpr int kPasses = (kFp8 ? 128 : 256) / kRowsPerPass;   // fp8 work tiles have at most 128 rows
     const int chunk = gt % kCpr, rbase = gt / kCpr;       // rows rbase + kRowsPerPass * j
     int islot = 0;
-    unsigned iph = 0, kiter = 0, phE = 0;                 // kiter: k-blocks of all GEMM tiles so far
+    unsigned iph = 0, kiter = 0;                          // kiter: k-blocks of all GEMM tiles so far
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 13))) break;
       const int kind = sc->info[islot].kind;
@@ -773,8 +803,14 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
       if (kind == kEnd) break;
       if (kind == kCombine) continue;
-      if (kind == kDown) {             // nothing to gather; only the stage index moves on
-        kiter += (unsigned)kblocks;
+      if (kind == kDown) {             // nothing to gather: hand every stage on empty-handed
+        bool failed = false;
+        for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
+          const int stage = (int)(kiter % kStages);
+          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kStages) & 1u) ^ 1u, 15))) { failed = true; break; }
+          mbar_arrive(&sc->fullA[stage]);
+        }
+        if (failed) break;
         continue;
       }
       const OpDev* op = &args.ops[slot];
@@ -788,12 +824,8 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       }
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
-        // The producer relays "stage free" for gate/up k-blocks through emptyA: that barrier
-        // advances only when this warp takes part, so its parity never aliases (a parity wait is
-        // only meaningful for a waiter within one phase of the barrier).
         const int stage = (int)(kiter % kStages);
-        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->emptyA[stage], (phE >> stage) & 1u, 14))) { fail = true; break; }
-        phE ^= 1u << stage;
+        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kStages) & 1u) ^ 1u, 14))) { fail = true; break; }
         const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
         const unsigned char* Xk = X + (size_t)kb * kRowBytes;
 #pragma unroll
