@@ -40,6 +40,7 @@ constexpr int kABytes = 2 * kAHalfBytes;               // up to 256 activation r
 constexpr int kBHalfBytes = 128 * kRowBytes;           // 128 weight rows of one k-block
 constexpr int kBBytes = 2 * kBHalfBytes;               // 256 weight rows per stage
 constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kMaxStages = 4;                          // fp8: four 48 KB stages, bf16: three 64 KB stages
 constexpr int kRing = 4;                               // tile-info ring depth
 constexpr int kAccCols = 256;                          // TMEM columns per accumulator
 constexpr int kEnd = -1;
@@ -52,7 +53,7 @@ struct TileInfo {
 };
 
 struct SharedCtl {
-  unsigned long long full[kStages], fullA[kStages], empty[kStages];
+  unsigned long long full[kMaxStages], fullA[kMaxStages], empty[kMaxStages];
   unsigned long long tfull[2], tempty[2];
   unsigned long long pfull[2], pempty[2];          // fp8: per-k-block partial products, two 256-column buffers
   unsigned long long xbar[4];                      // fp8: amax exchange between the two warps of a quadrant
@@ -65,6 +66,10 @@ struct SharedCtl {
   int cls_slot[2][kMaxOps];
   int cls_free[2][kMaxOps];        // 1: the op has no ready word and no predecessor
   unsigned cum[2][kMaxOps + 1];
+#ifdef MOE_TIMING_PROBE
+  int dbg_e;
+  int dbg_w[8];
+#endif
 };
 
 constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(SharedCtl);
@@ -363,35 +368,22 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
   float acc[128];                                 // [half][64]
 #pragma unroll
   for (int i = 0; i < 128; ++i) acc[i] = 0.f;
-  float4 vx = make_float4(0.f, 0.f, 0.f, 0.f), v0 = vx, v1 = vx;   // scales of four k-blocks at a time
+  // scales of the next k-block are loaded one k-block ahead (three scalars in flight)
+  float nfx = 0.f, nw0 = 0.f, nw1 = 0.f;
+  if (ti.kblocks > 0) { nfx = sx[0]; nw0 = sw0[0]; nw1 = sw1[0]; }
   for (int kb = 0; kb < ti.kblocks; ++kb) {
-    if ((kb & 3) == 0) {
-      // the scale rows are contiguous over k-blocks; their lengths (H/128, I/128) are multiples of 4
-      // for the supported shapes, else fall back to scalar loads
-      if (((ti.kblocks & 3) == 0)) {
-        vx = *reinterpret_cast<const float4*>(sx + kb);
-        v0 = *reinterpret_cast<const float4*>(sw0 + kb);
-        v1 = *reinterpret_cast<const float4*>(sw1 + kb);
-      } else {
-        float tx[4], t0[4], t1[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int kk = min(kb + i, ti.kblocks - 1);
-          tx[i] = sx[kk]; t0[i] = sw0[kk]; t1[i] = sw1[kk];
-        }
-        vx = make_float4(tx[0], tx[1], tx[2], tx[3]);
-        v0 = make_float4(t0[0], t0[1], t0[2], t0[3]);
-        v1 = make_float4(t1[0], t1[1], t1[2], t1[3]);
-      }
-    }
-    const int sub = kb & 3;
-    const float fx = sub == 0 ? vx.x : (sub == 1 ? vx.y : (sub == 2 ? vx.z : vx.w));
-    const float s0 = fx * (sub == 0 ? v0.x : (sub == 1 ? v0.y : (sub == 2 ? v0.z : v0.w)));
-    const float s1 = fx * (sub == 0 ? v1.x : (sub == 1 ? v1.y : (sub == 2 ? v1.z : v1.w)));
+    const float s0 = nfx * nw0, s1 = nfx * nw1;
+    if (kb + 1 < ti.kblocks) { nfx = sx[kb + 1]; nw0 = sw0[kb + 1]; nw1 = sw1[kb + 1]; }
     const int pb = kb & 1;
+#ifdef MOE_TIMING_PROBE
+    const long long e0 = clock64();
+#endif
     if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->pfull[pb], (eph >> pb) & 1u, 19))) return false;
     eph ^= 1u << pb;
     tc_fence_after();
+#ifdef MOE_TIMING_PROBE
+    const long long e1 = clock64();
+#endif
     // eight 16-column chunks (four per half); the load of chunk c+1 is in flight while chunk c
     // is multiplied in
     const unsigned pbase = lane_addr + (unsigned)(pb * 256 + ch * 64);
@@ -407,7 +399,14 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
         acc[cc * 16 + i] = fmaf(__uint_as_float(p[cc & 1][i]), s, acc[cc * 16 + i]);
     }
     tc_fence_before();
-    mbar_arrive(&sc->pempty[pb]);                 // the partial buffer may be overwritten
+    __syncwarp();                                 // every lane's TMEM loads have completed
+    if (lane == 0) mbar_arrive(&sc->pempty[pb]); // one arrival per warp: the partial buffer may be overwritten
+#ifdef MOE_TIMING_PROBE
+    if (blockIdx.x == 7 && lane == 0 && sc->dbg_w[warp - 8] < 2048) {
+      long long* pp = a.dbg + 16384 + (size_t)(warp - 8) * 8192 + (size_t)sc->dbg_w[warp - 8]++ * 4;
+      pp[0] = e0; pp[1] = e1; pp[2] = clock64(); pp[3] = ti.kind * 1000 + kb;
+    }
+#endif
   }
   // the accumulator is complete
   if (g1) {
@@ -479,15 +478,24 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
                                                               RunHead* rh) {
   constexpr int kKb = kFp8 ? 128 : kBlockK;     // K elements per stage (128 bytes per row either way)
   constexpr int kEl = kFp8 ? 1 : 2;             // bytes per element
+  // fp8 tiles have at most 128 rows: a stage holds 128 activation rows + 256 weight rows
+  constexpr int kNS = kFp8 ? 4 : 3;
+  constexpr int kBOff = kFp8 ? kAHalfBytes : kABytes;
+  constexpr int kSB = kBOff + kBBytes;
   extern __shared__ unsigned char smem_raw[];
   unsigned char* stages = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  SharedCtl* sc = reinterpret_cast<SharedCtl*>(stages + (size_t)kStages * kStageBytes);
+  SharedCtl* sc = reinterpret_cast<SharedCtl*>(stages + (size_t)kNS * kSB);
+  static_assert(kNS * kSB == 3 * (kABytes + kBBytes), "ring size");
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   Ctx c{&args, &args.g->status};
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
+#ifdef MOE_TIMING_PROBE
+    sc->dbg_e = 0;
+    for (int i = 0; i < 8; ++i) sc->dbg_w[i] = 0;
+#endif
+    for (int s = 0; s < kNS; ++s) {
       mbar_init(&sc->full[s], 1);
       mbar_init(&sc->fullA[s], kGatherThreads);
       mbar_init(&sc->empty[s], 1);
@@ -498,7 +506,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     }
     for (int s = 0; s < 2; ++s) {
       mbar_init(&sc->pfull[s], 1);
-      mbar_init(&sc->pempty[s], 256);
+      mbar_init(&sc->pempty[s], 8);
     }
     for (int s = 0; s < 4; ++s) mbar_init(&sc->xbar[s], 64);
     // a ring slot is released by the MMA warp, the committer and each gather warp
@@ -591,15 +599,15 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #ifdef MOE_TIMING_PROBE
             if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 0] = clock64();
 #endif
-            unsigned char* sA = stages + (size_t)stage * kStageBytes;
-            unsigned char* sB = sA + kABytes;
+            unsigned char* sA = stages + (size_t)stage * kSB;
+            unsigned char* sB = sA + kBOff;
             mbar_expect_tx(&sc->full[stage], tx);
             tma_tile_2d(sB, tmw, kb * kKb, wrow0, &sc->full[stage]);
             tma_tile_2d(sB + kBHalfBytes, tmw, kb * kKb, wrow1, &sc->full[stage]);
             if (!g1) tma_tile_2d(sA, tma, kb * kKb, ti.row0, &sc->full[stage]);
           }
           __syncwarp();
-          if (++stage == kStages) { stage = 0; ph ^= 1u; }
+          if (++stage == kNS) { stage = 0; ph ^= 1u; }
           if (kb == claim_at)              // claim ahead (never blocks here)
             have_nx = claim_once(c, sc, rh, lane, nx, nx_need_ready) == 1;
           if (have_nx && !nx_published && kb > claim_at && kb >= ti.kblocks - kPublishLead) {
@@ -646,7 +654,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     int dbg_i = 0, dbg_t = 0;
 #endif
     int stage = 0, islot = 0;
-    unsigned ph = 0, iph = 0, aph[2] = {0, 0}, phA = 0, pph = 0;
+    unsigned ph = 0, iph = 0, aph[2] = {0, 0}, pph = 0;
     AccUse accs;
     while (true) {
       if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->ifull[islot], iph, 6))) break;
@@ -689,9 +697,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #endif
             if (lane == 0) {
               fence_async_proxy_smem();
-              const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
+              const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
               const unsigned long long ad = umma_desc(sA, kRowBytes);
-              const unsigned long long bd = umma_desc(sA + kABytes, kRowBytes);
+              const unsigned long long bd = umma_desc(sA + kBOff, kRowBytes);
 #pragma unroll
               for (int k4 = 0; k4 < 4; ++k4)              // 32 e4m3 elements (32 bytes) per step
                 tc_mma_f8(tmem + (unsigned)(pb * 256), ad + 2ull * k4, bd + 2ull * k4, kIdescF8, k4 ? 1u : 0u);
@@ -701,7 +709,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
             __syncwarp();
           }
           if (fail) break;
-          if (++stage == kStages) { stage = 0; ph ^= 1u; }
+          if (++stage == kNS) { stage = 0; ph ^= 1u; }
         }
         if (fail) break;
       } else if (kind != kCombine) {
@@ -732,8 +740,8 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
             if (blockIdx.x == 7 && dbg_i < 4096) { args.dbg[dbg_i * 4 + 1] = clock64(); args.dbg[dbg_i * 4 + 2] = kind * 1000 + rows; }
 #endif
             fence_async_proxy_smem();                    // cp.async-written rows -> tensor core reads
-            const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
-            const unsigned long long ad = umma_desc(sA, kRowBytes), bd = umma_desc(sA + kABytes, kRowBytes);
+            const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
+            const unsigned long long ad = umma_desc(sA, kRowBytes), bd = umma_desc(sA + kBOff, kRowBytes);
 #pragma unroll
             for (int k4 = 0; k4 < kBlockK / 16; ++k4)   // +32 bytes along K per step (>>4 = 2)
               tc_mma_bf16(d0, ad + 2ull * k4, bd + 2ull * k4, kIdesc, (kb | k4) ? 1u : 0u);
@@ -746,8 +754,8 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #endif
           }
           if (lane == 0) {
-            const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
-            const unsigned long long bd = umma_desc(sA + kABytes, kRowBytes);
+            const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
+            const unsigned long long bd = umma_desc(sA + kBOff, kRowBytes);
             if (pair) {                                  // rows 128..255 against the same weight tile
               const unsigned long long ad1 = umma_desc(sA + kAHalfBytes, kRowBytes);
 #pragma unroll
@@ -760,7 +768,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #endif
           }
           __syncwarp();
-          if (++stage == kStages) { stage = 0; ph ^= 1u; }
+          if (++stage == kNS) { stage = 0; ph ^= 1u; }
         }
         if (fail) break;
         if (lane == 0) {                                 // accumulator(s) complete
@@ -806,9 +814,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (kind == kDown) {             // nothing to gather: hand every stage on empty-handed
         bool failed = false;
         for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
-          const int stage = (int)(kiter % kStages);
-          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kStages) & 1u) ^ 1u, 15))) { failed = true; break; }
-          mbar_arrive(&sc->fullA[stage]);
+          const int stage = (int)(kiter % kNS);
+          if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kNS) & 1u) ^ 1u, 15))) { failed = true; break; }
+          if (lane == 0) mbar_arrive_n(&sc->fullA[stage], 32);   // the whole warp's share in one arrival
         }
         if (failed) break;
         continue;
@@ -824,9 +832,9 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       }
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
-        const int stage = (int)(kiter % kStages);
-        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kStages) & 1u) ^ 1u, 14))) { fail = true; break; }
-        const unsigned sA = smem_u32(stages + (size_t)stage * kStageBytes);
+        const int stage = (int)(kiter % kNS);
+        if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kNS) & 1u) ^ 1u, 14))) { fail = true; break; }
+        const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
         const unsigned char* Xk = X + (size_t)kb * kRowBytes;
 #pragma unroll
         for (int j = 0; j < kPasses; ++j) {
@@ -964,7 +972,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           mbar_arrive(&sc->tempty[b]);            // accumulator may be overwritten
 #ifdef MOE_TIMING_PROBE
           if (blockIdx.x == 7 && warp == 8 && lane == 0 && dbg_e < 1024) {
-            long long* pp = args.dbg + 12288 * 4 + (size_t)dbg_e++ * 4;
+            long long* pp = args.dbg + 12288 * 4 + (size_t)sc->dbg_e++ * 4;
             pp[0] = te0; pp[1] = te1; pp[2] = clock64(); pp[3] = ti.kind * 1000 + ti.rows + b * 100000;
           }
 #endif
