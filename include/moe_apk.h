@@ -97,7 +97,7 @@ typedef struct {
   int32_t slot;      /* op slot                                                           */
   int32_t tile;      /* index in the op's tile list                                       */
   int16_t cls, kind; /* class; 0 = gate/up GEMM + SwiGLU, 1 = down GEMM, 2 = combine      */
-  int16_t cta, sm;   /* CTA index and SM id that ran it                                   */
+  int16_t cta, sm;   /* CTA index and SM id that ran it (first CTA of a pair)                */
 } moe_tile_rec_t;
 
 /* Bytes of device workspace moe_create needs for this configuration. */
@@ -178,6 +178,14 @@ int moe_plan_static(const int32_t* topk_ids, int32_t n_tokens, int32_t top_k, in
 
 /* Multiprocessor count of the context's device (the default persistent grid). */
 int moe_sm_count(moe_ctx_t* ctx);
+
+/* How many CTAs work on one tile: 2 when the context runs bf16 on an even grid (tiles are
+ * then claimed and run by pairs of CTAs on neighbouring SMs, one tcgen05 MMA spanning both),
+ * else 1.  The claiming unit of Section 4.2 is that group: the decode budget of
+ * moe_set_budget still counts CTAs (a pair is inside the budget when its first CTA is), and
+ * tile records carry the CTA index and SM id of the group's first CTA.  Setting
+ * MOE_APK_SINGLE_CTA=1 in the environment before moe_create keeps every context at 1. */
+int moe_ctas_per_tile(moe_ctx_t* ctx);
 
 const char* moe_strerror(int code);
 

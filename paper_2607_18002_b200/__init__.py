@@ -28,7 +28,7 @@ MOE_TILE_M = 128
 
 EXPORTS = ("moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_run",
            "moe_combine", "moe_set_budget", "moe_status", "moe_footprint",
-           "moe_read_tile_table", "moe_read_tile_log", "moe_sm_count", "moe_strerror",
+           "moe_read_tile_table", "moe_read_tile_log", "moe_sm_count", "moe_ctas_per_tile", "moe_strerror",
            "moe_plan_static")
 MOE_PLAN_STATIC_MAX_ROWS, MOE_PLAN_STATIC_MAX_EXPERTS = 32768, 256
 
@@ -95,6 +95,7 @@ def lib() -> C.CDLL:
         L.moe_read_tile_log.argtypes = [vp, vp, C.c_int, C.POINTER(C.c_int)]
         L.moe_plan_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
         L.moe_sm_count.argtypes = [vp]
+        L.moe_ctas_per_tile.argtypes = [vp]
         L.moe_strerror.argtypes = [C.c_int]
         L.moe_strerror.restype = C.c_char_p
         for name in EXPORTS:
@@ -193,6 +194,10 @@ def moe_plan_static(topk_ids_ptr: int, n_tokens: int, top_k: int, n_experts: int
 
 def moe_sm_count(ctx: int) -> int:
     return int(lib().moe_sm_count(C.c_void_p(ctx)))
+
+
+def moe_ctas_per_tile(ctx: int) -> int:
+    return int(lib().moe_ctas_per_tile(C.c_void_p(ctx)))
 
 
 # ------------------------------------------------------------------ conveniences
@@ -313,3 +318,7 @@ class Context:
     @property
     def sm_count(self) -> int:
         return moe_sm_count(self.ctx)
+
+    @property
+    def ctas_per_tile(self) -> int:
+        return moe_ctas_per_tile(self.ctx)

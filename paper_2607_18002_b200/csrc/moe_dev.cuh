@@ -63,6 +63,7 @@ struct __align__(128) OpDev {
   CUtensorMap tm_w2;    // [E*H, I]    box {64, 128} down weights
   CUtensorMap tm_a128;  // [Rmax, I]   box {64, 128}
   CUtensorMap tm_a256;  // [Rmax, I]   box {64, 256}
+  CUtensorMap tm_w1h;   // [E*2I, H]   box {64, 64}  gate/up weights, half-height box (CTA-pair kernel)
   int cls, n_tokens, n_rows, after_op;
   const void* x;
   const float* x_scale;

@@ -14,6 +14,8 @@ cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, in
 cudaError_t launch_combine(const OpDev* d_op, int T, int k, int H, cudaStream_t stream);
 cudaError_t prepare_run_kernel();
 cudaError_t launch_run(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream);
+cudaError_t prepare_pair_kernel();
+cudaError_t launch_pair(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream);
 }  // namespace moe
 
 using namespace moe;
@@ -90,6 +92,7 @@ struct moe_ctx {
   Layout L;
   unsigned char* ws;
   int n_ctas, sm_count;
+  bool pair_kernel;             // bf16 on an even grid: tiles run on CTA pairs (cta_group::2)
   EncodeTiledFn encode;
   moe_op_t ops[kMaxOps];
   bool planned[kMaxOps];
@@ -177,7 +180,7 @@ int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_c
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
       qres != cudaDriverEntryPointSuccess || !fn)
     return MOE_ECUDA;
-  if (prepare_run_kernel() != cudaSuccess) return MOE_ECUDA;
+  if (prepare_run_kernel() != cudaSuccess || prepare_pair_kernel() != cudaSuccess) return MOE_ECUDA;
   moe_ctx* ctx = new (std::nothrow) moe_ctx();
   if (!ctx) return MOE_ENOSPC;
   ctx->cfg = *cfg;
@@ -186,6 +189,10 @@ int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_c
   ctx->ws = static_cast<unsigned char*>(dev_workspace);
   ctx->sm_count = sms;
   ctx->n_ctas = cfg->n_ctas > 0 ? cfg->n_ctas : sms;
+  // MOE_APK_SINGLE_CTA=1 in the environment keeps bf16 on the one-CTA-per-tile kernel (for comparisons)
+  const char* single = getenv("MOE_APK_SINGLE_CTA");
+  ctx->pair_kernel = cfg->dtype == MOE_DTYPE_BF16 && ctx->n_ctas >= 2 && ctx->n_ctas % 2 == 0 &&
+                     !(single && single[0] == '1');
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   memset(ctx->planned, 0, sizeof(ctx->planned));
   memset(ctx->uploaded, 0, sizeof(ctx->uploaded));
@@ -201,6 +208,7 @@ int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_c
 void moe_destroy(moe_ctx_t* ctx) { delete ctx; }
 
 int moe_sm_count(moe_ctx_t* ctx) { return ctx ? ctx->sm_count : MOE_EINVAL; }
+int moe_ctas_per_tile(moe_ctx_t* ctx) { return ctx ? (ctx->pair_kernel ? 2 : 1) : MOE_EINVAL; }
 
 int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   if (!ctx || !op) return MOE_EINVAL;
@@ -254,6 +262,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
       if (!rc) rc = make_map(ctx, &h.tm_a128, h.A, (size_t)L.max_rows, (size_t)c.inter, 128);
       if (!rc) rc = make_map(ctx, &h.tm_a256, h.A, (size_t)L.max_rows, (size_t)c.inter, 256);
       if (!rc) rc = make_map(ctx, &h.tm_w1, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 128);
+      if (!rc) rc = make_map(ctx, &h.tm_w1h, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 64);
       if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
       if (rc) return rc;
     }
@@ -305,7 +314,9 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
 #endif
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
-  if (launch_run(a, ctx->rh(), ctx->n_ctas, st) != cudaSuccess) return MOE_ECUDA;
+  const cudaError_t le = ctx->pair_kernel ? launch_pair(a, ctx->rh(), ctx->n_ctas, st)
+                                          : launch_run(a, ctx->rh(), ctx->n_ctas, st);
+  if (le != cudaSuccess) return MOE_ECUDA;
   return MOE_OK;
 }
 

@@ -35,6 +35,18 @@ __device__ __forceinline__ bool mbar_try(void* bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
+// non-blocking test of a phase (try_wait may suspend the thread for a while)
+__device__ __forceinline__ bool mbar_test(void* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
 __device__ __forceinline__ void tma_tile_2d(void* dst, const CUtensorMap* tm, int x, int y,
                                             void* bar) {
   asm volatile(
@@ -138,6 +150,11 @@ __device__ __forceinline__ void cp_async_16(unsigned dst_smem, const void* src) 
 __device__ __forceinline__ void cp_async_arrive_noinc(void* bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int kPending>
+__device__ __forceinline__ void cp_async_wait_group() {
+  asm volatile("cp.async.wait_group %0;" ::"n"(kPending) : "memory");
+}
 __device__ __forceinline__ void cp_async_wait_all() {
   asm volatile("cp.async.wait_all;" ::: "memory");
 }
@@ -178,4 +195,148 @@ __device__ __forceinline__ unsigned long long umma_desc(unsigned saddr, unsigned
 constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17) | ((128u >> 4) << 24);
 
 
+
+// ------------------------------------------------------------------ CTA pairs (cluster of two)
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {      // every thread of both CTAs
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// shared::cluster address of the same shared-memory object in CTA `rank` of the cluster
+__device__ __forceinline__ unsigned map_to_cta(const void* p, unsigned rank) {
+  unsigned r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(unsigned cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_cluster(unsigned cluster_addr, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.release.cluster.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+// the same two without cluster-scope release: for pipeline barriers whose data moves by TMA or cp.async
+__device__ __forceinline__ void mbar_arrive_remote(unsigned cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_remote(unsigned cluster_addr, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;" ::"r"(cluster_addr), "r"(bytes) : "memory");
+}
+// wait that synchronises with arrivals made by the other CTA of the pair
+__device__ __forceinline__ bool mbar_try_cluster(void* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ void st_cluster_v4(unsigned cluster_addr, uint4 v) {
+  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(cluster_addr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+// tiled TMA load by either CTA of a pair; the transaction bytes go to the barrier at `bar_cluster_addr`
+// (the pair leader's), the data to this CTA's own shared memory
+__device__ __forceinline__ void tma_tile_2d_pair(void* dst, const CUtensorMap* tm, int x, int y, unsigned bar_cluster_addr) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(smem_u32(dst)),
+      "l"(reinterpret_cast<unsigned long long>(tm)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+// one MMA of the pair: M = 256 or 128 rows split over the two CTAs, both halves of B read from the two CTAs
+__device__ __forceinline__ void tc_mma2_bf16(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                             unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+// arrives on the barrier at the same shared-memory offset in both CTAs once the pair's MMAs so far retire
+__device__ __forceinline__ void tc_commit_pair(void* bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
+}
+
+// ---- warp-uniform issue: the whole warp executes these, one elected lane issues the instruction.
+// Their operands then stay warp-uniform for the compiler (no per-thread staging of descriptors),
+// which keeps the issue loops of the MMA and producer warps short.
+__device__ __forceinline__ void tc_mma2_bf16_elect(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                                   unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p, e;\n\t.reg .b32 r;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "@e tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair_elect(void* bar) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\t.reg .b32 r;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}" ::"r"(smem_u32(bar)),
+      "h"((unsigned short)3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_tile_2d_pair_elect(unsigned dst_smem, const CUtensorMap* tm, int x, int y, unsigned bar_cluster_addr) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\t.reg .b32 r;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "@e cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];\n\t}" ::"r"(dst_smem),
+      "l"(reinterpret_cast<unsigned long long>(tm)), "r"(bar_cluster_addr), "r"(x), "r"(y)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx_addr_elect(unsigned cluster_addr, unsigned bytes) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\t.reg .b32 r;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "@e mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;\n\t}" ::"r"(cluster_addr), "r"(bytes)
+      : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_n_elect(void* bar, unsigned n) {
+  asm volatile(
+      "{\n\t.reg .pred e;\n\t.reg .b32 r;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "@e mbarrier.arrive.shared::cta.b64 _, [%0], %1;\n\t}" ::"r"(smem_u32(bar)), "r"(n)
+      : "memory");
+}
+
+// All loads and barrier arrivals of one k-block by one CTA of a pair, as ONE instruction group under a
+// single election: expect_tx on the leader's stage barrier, up to two weight boxes, up to two
+// activation boxes, the stand-in arrivals (tiles without a gather) and the go-ahead for the gather warps.
+// Flags select what is issued; everything is warp-uniform.
+__device__ __forceinline__ void pair_issue_kblock(unsigned bar, unsigned tx, unsigned standin_bar, unsigned standin_n,
+                                                  unsigned sB, const CUtensorMap* tmw, int x, int wy0, int wy1, unsigned has_w1,
+                                                  unsigned sA, const CUtensorMap* tma, int ay, unsigned a_boxes,
+                                                  unsigned go_bar, unsigned has_go) {
+  asm volatile(
+      "{\n\t.reg .pred e, pw1, pa1, pa2, pgo, pst;\n\t.reg .b32 r, sB1, sA1, ay1;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "setp.ne.and.b32 pw1, %9, 0, e;\n\t"
+      "setp.ge.and.u32 pa1, %13, 1, e;\n\t"
+      "setp.ge.and.u32 pa2, %13, 2, e;\n\t"
+      "setp.ne.and.b32 pgo, %15, 0, e;\n\t"
+      "setp.ne.and.b32 pst, %3, 0, e;\n\t"
+      "add.u32 sB1, %4, 8192;\n\t"
+      "add.u32 sA1, %10, 4096;\n\t"
+      "add.s32 ay1, %12, 32;\n\t"
+      "@e mbarrier.arrive.expect_tx.shared::cluster.b64 _, [%0], %1;\n\t"
+      "@pst mbarrier.arrive.shared::cta.b64 _, [%2], %3;\n\t"
+      "@e cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%4], [%5, {%6, %7}], [%0];\n\t"
+      "@pw1 cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [sB1], [%5, {%6, %8}], [%0];\n\t"
+      "@pa1 cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%10], [%11, {%6, %12}], [%0];\n\t"
+      "@pa2 cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [sA1], [%11, {%6, ay1}], [%0];\n\t"
+      "@pgo mbarrier.arrive.shared::cta.b64 _, [%14];\n\t}"
+      ::"r"(bar), "r"(tx), "r"(standin_bar), "r"(standin_n),
+        "r"(sB), "l"(reinterpret_cast<unsigned long long>(tmw)), "r"(x), "r"(wy0), "r"(wy1), "r"(has_w1),
+        "r"(sA), "l"(reinterpret_cast<unsigned long long>(tma)), "r"(ay), "r"(a_boxes),
+        "r"(go_bar), "r"(has_go)
+      : "memory");
+}
 }  // namespace moe

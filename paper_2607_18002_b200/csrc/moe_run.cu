@@ -29,6 +29,7 @@
 // kernel records MOE_ETIMEOUT, raises the abort word, and all CTAs drain and return.
 #include "moe_combine.cuh"
 #include "moe_ptx.cuh"
+#include "moe_sched.cuh"
 #include <cuda_fp8.h>
 
 namespace moe {
@@ -41,16 +42,7 @@ constexpr int kBHalfBytes = 128 * kRowBytes;           // 128 weight rows of one
 constexpr int kBBytes = 2 * kBHalfBytes;               // 256 weight rows per stage
 constexpr int kStageBytes = kABytes + kBBytes;
 constexpr int kMaxStages = 4;                          // fp8: four 48 KB stages, bf16: three 64 KB stages
-constexpr int kRing = 4;                               // tile-info ring depth
 constexpr int kAccCols = 256;                          // TMEM columns per accumulator
-constexpr int kEnd = -1;
-constexpr int kClaimAt = 2;                             // claim the next tile after this k-block
-constexpr int kPublishLead = 5;                         // try to hand the next tile on from this many k-blocks before the end
-
-struct TileInfo {
-  int kind, slot, tile, m, row0, rows, n, kblocks, expert, cls;
-  unsigned long long t_claim;
-};
 
 struct SharedCtl {
   unsigned long long full[kMaxStages], fullA[kMaxStages], empty[kMaxStages];
@@ -62,10 +54,7 @@ struct SharedCtl {
   TileInfo info[kRing];
   unsigned tmem_base;
   alignas(16) unsigned char epi_scratch[8][2048];   // per epilogue warp: 32 rows x 64 bytes
-  int n_cls[2];
-  int cls_slot[2][kMaxOps];
-  int cls_free[2][kMaxOps];        // 1: the op has no ready word and no predecessor
-  unsigned cum[2][kMaxOps + 1];
+  QueueTables qt;
 #ifdef MOE_TIMING_PROBE
   int dbg_e;
   int dbg_w[8];
@@ -73,264 +62,6 @@ struct SharedCtl {
 };
 
 constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(SharedCtl);
-
-// ------------------------------------------------------------------ bounded waits
-struct Ctx {
-  const RunArgs* a;
-  Status* st;
-};
-
-__device__ __forceinline__ bool aborted(const Ctx& c) { return ld_volatile(&c.st->abort) != 0; }
-
-// where: a small code telling which wait gave up (reported in detail[0])
-__device__ __noinline__ bool mbar_wait_slow(const Ctx& c, void* bar, unsigned parity, int where) {
-  unsigned long long t0 = 0;
-  for (unsigned it = 1;; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if ((it & 63u) == 0) {
-      if (aborted(c)) return false;
-      const unsigned long long now = gtime_ns();
-      if (t0 == 0) t0 = now;
-      else if ((long long)(now - t0) > c.a->wait_ns) {
-        report(c.st, MOE_ETIMEOUT, where, (int)blockIdx.x, (int)threadIdx.x, (int)parity);
-        return false;
-      }
-    }
-  }
-}
-__device__ __forceinline__ bool mbar_wait(const Ctx& c, void* bar, unsigned parity, int where) {
-  if (mbar_try(bar, parity)) return true;
-  return mbar_wait_slow(c, bar, parity, where);
-}
-
-// the same wait without any function call: for code that keeps many registers live across it
-__device__ __forceinline__ bool mbar_wait_inline(const Ctx& c, void* bar, unsigned parity, int where) {
-  unsigned long long t0 = 0;
-  for (unsigned it = 0;; ++it) {
-    if (mbar_try(bar, parity)) return true;
-    if ((it & 63u) == 63u) {
-      if (aborted(c)) return false;
-      const unsigned long long now = gtime_ns();
-      if (t0 == 0) t0 = now;
-      else if ((long long)(now - t0) > c.a->wait_ns) {
-        if (atomicCAS(&c.st->code, 0, MOE_ETIMEOUT) == 0) {
-          c.st->detail[0] = where; c.st->detail[1] = (int)blockIdx.x;
-          c.st->detail[2] = (int)threadIdx.x; c.st->detail[3] = (int)parity;
-        }
-        __threadfence();
-        atomicExch(&c.st->abort, 1);
-        return false;
-      }
-    }
-  }
-}
-
-// spin until *p >= target (acquire); one thread
-__device__ __noinline__ bool wait_counter(const Ctx& c, const int* p, int target, int where) {
-  unsigned long long t0 = 0;
-  for (unsigned it = 0;; ++it) {
-    if (ld_acquire(p) >= target) return true;
-    if (it > 16) __nanosleep(64);
-    if ((it & 63u) == 63u) {
-      if (aborted(c)) return false;
-      const unsigned long long now = gtime_ns();
-      if (t0 == 0) t0 = now;
-      else if ((long long)(now - t0) > c.a->wait_ns) {
-        report(c.st, MOE_ETIMEOUT, where, (int)blockIdx.x, target, ld_acquire(p));
-        return false;
-      }
-    }
-  }
-}
-
-// ------------------------------------------------------------------ queues
-__device__ __forceinline__ int op_total_tiles(const OpDev* op, int fuse) {
-  return op->plan->n_gemm_tiles + (fuse ? op->plan->n_comb_tiles : 0);
-}
-
-__device__ inline bool op_ready(const RunArgs* a, const OpDev* op) {
-  if (op->ready != nullptr && ld_acquire_sys(op->ready) == 0) return false;
-  if (op->after_op >= 0 && ld_acquire(&a->ops[op->after_op].run->done) == 0) return false;
-  return true;
-}
-
-// Claim by the whole producer warp.  1: claimed (ti filled), 0: queue exhausted, -1: the op
-// at the head of the queue is not ready.  The head is only peeked before the fetch-add, so no
-// CTA can be starved by others (a compare-and-swap loop starves the SMs far from the counter);
-// the price is that a ticket can land just past an op boundary, in an op that is not ready
-// yet -- the caller then waits for it (bounded), holding only tickets whose predecessors in
-// the queue are all claimed already.
-__device__ inline int try_claim(const RunArgs* a, SharedCtl* sc, RunHead* rh, int cls, unsigned h,
-                                int lane, TileInfo& ti, bool& need_ready) {
-  const int n = sc->n_cls[cls];
-  if (n == 0) return 0;
-  const unsigned total = sc->cum[cls][n];
-  h = __shfl_sync(0xffffffffu, h, 0);       // one peek for the whole warp: lanes index entries by it
-  if (h >= total) return 0;
-  int i = 0;
-  while (h >= sc->cum[cls][i + 1]) ++i;
-  int slot = sc->cls_slot[cls][i];
-  const OpDev* op = &a->ops[slot];
-  if (!sc->cls_free[cls][i] && !op_ready(a, op)) return -1;
-  // the 32 entries from the head on are fetched while the fetch-add is in flight
-  const unsigned base = h - sc->cum[cls][i];
-  const unsigned n_op = sc->cum[cls][i + 1] - sc->cum[cls][i];
-  int4 e = make_int4(0, 0, 0, 0);
-  if (base + lane < n_op) e = op->tile_list[base + lane];
-  unsigned t = 0;
-  if (lane == 0) t = atomicAdd(&rh->heads[cls], 1u);
-  t = __shfl_sync(0xffffffffu, t, 0);
-  if (t >= total) return 0;
-  need_ready = false;
-  if (t >= sc->cum[cls][i + 1]) {          // past the op boundary: a later op of the class
-    while (t >= sc->cum[cls][i + 1]) ++i;
-    slot = sc->cls_slot[cls][i];
-    op = &a->ops[slot];
-    need_ready = !sc->cls_free[cls][i];
-  }
-  const unsigned local = t - sc->cum[cls][i];
-  const unsigned d = t - h;
-  const bool hit = !need_ready && d < 32u;
-  int4 got;
-  got.x = __shfl_sync(0xffffffffu, e.x, hit ? d : 0);
-  got.y = __shfl_sync(0xffffffffu, e.y, hit ? d : 0);
-  got.z = __shfl_sync(0xffffffffu, e.z, hit ? d : 0);
-  got.w = __shfl_sync(0xffffffffu, e.w, hit ? d : 0);
-  if (!hit) got = op->tile_list[local];
-  ti.kind = entry_kind(got);
-  ti.n = entry_n(got);
-  ti.m = entry_m(got);
-  ti.row0 = got.y;
-  ti.rows = got.z;
-  ti.expert = got.w;
-  ti.slot = slot;
-  ti.tile = (int)local;
-  ti.cls = cls;
-  ti.kblocks = ti.kind == kCombine ? 0 : (ti.kind == kGateUp ? a->H : a->I) / a->kb_elems;
-  return 1;
-}
-
-// One pass of the decision at a tile boundary (whole producer warp): 1 = claimed, 0 = both
-// queues exhausted, -1 = something exists but is not ready yet.  The abort word, the budget
-// word and both queue heads are loaded together (one round trip), then at most one
-// fetch-add per class.
-__device__ inline int claim_once(const Ctx& c, SharedCtl* sc, RunHead* rh, int lane, TileInfo& ti,
-                                 bool& need_ready) {
-  const RunArgs* a = c.a;
-  const int ab = ld_volatile(&c.st->abort);
-  const int q = ld_volatile(&a->g->budget);
-  const unsigned h0 = *reinterpret_cast<volatile unsigned*>(&rh->heads[0]);
-  const unsigned h1 = *reinterpret_cast<volatile unsigned*>(&rh->heads[1]);
-  if (ab != 0) return 0;
-  const int first = ((int)blockIdx.x < q) ? MOE_CLASS_DECODE : MOE_CLASS_PREFILL;
-  need_ready = false;
-  const int r1 = try_claim(a, sc, rh, first, first == 0 ? h0 : h1, lane, ti, need_ready);
-  int r2 = 0;
-  if (r1 != 1) r2 = try_claim(a, sc, rh, 1 - first, first == 0 ? h1 : h0, lane, ti, need_ready);
-  if (r1 == 1 || r2 == 1) {
-    ti.t_claim = gtime_ns();
-    return 1;
-  }
-  return (r1 == 0 && r2 == 0) ? 0 : -1;
-}
-
-// A ticket that landed in an op that is not ready yet: wait for it (bounded).
-__device__ inline bool wait_op_ready(const Ctx& c, int lane, const TileInfo& ti) {
-  const RunArgs* a = c.a;
-  const unsigned long long w0 = gtime_ns();
-  while (!op_ready(a, &a->ops[ti.slot])) {
-    __nanosleep(256);
-    if (aborted(c)) return false;
-    if ((long long)(gtime_ns() - w0) > a->wait_ns) {
-      if (lane == 0) report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, ti.slot, ti.tile);
-      return false;
-    }
-  }
-  return true;
-}
-
-// Blocking form: waits (bounded) while an op exists that is not ready.  Returns with
-// ti.kind == kEnd when nothing is left (or the run was aborted).
-__device__ inline void claim_next(const Ctx& c, SharedCtl* sc, RunHead* rh, int lane, TileInfo& ti,
-                                  bool& need_ready) {
-  unsigned long long t0 = 0;
-  for (unsigned it = 0;; ++it) {
-    const int r = claim_once(c, sc, rh, lane, ti, need_ready);
-    if (r == 1) return;
-    if (r == 0) break;
-    __nanosleep(256);                         // an op exists but is not ready yet
-    if ((it & 15u) == 15u) {
-      const unsigned long long now = gtime_ns();
-      if (t0 == 0) t0 = now;
-      else if ((long long)(now - t0) > c.a->wait_ns) {
-        if (lane == 0) report(c.st, MOE_ETIMEOUT, 1, (int)blockIdx.x, 0, 0);
-        break;
-      }
-    }
-  }
-  ti.kind = kEnd;
-}
-
-// Publishing a finished tile: dependency counter, op completion, done word, log.
-// Called by one thread after all writers of the tile have fenced and synchronised.
-__device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti) {
-  const RunArgs* a = c.a;
-  OpDev* op = &a->ops[ti.slot];
-  __threadfence();
-  fence_async_proxy();
-  const unsigned long long t_commit = a->log_cap > 0 ? gtime_ns() : 0ull;   // before it is published
-  if (ti.kind == kGateUp) atomicAdd(&op->g1_done[ti.m], 1);
-  if (ti.kind != kCombine) atomicAdd(&op->run->gemm_done, 1);
-  const int done = atomicAdd(&op->run->tiles_done, 1) + 1;
-  if (done == op_total_tiles(op, a->fuse_combine)) {
-    __threadfence();
-    atomicExch(&op->run->done, 1);
-    if (op->done != nullptr) st_release_sys(op->done, 1u);
-  }
-  if (a->log_cap > 0) {
-    const unsigned idx = atomicAdd(&rh->log_count, 1u);
-    if (idx < (unsigned)a->log_cap) {
-      moe_tile_rec_t r;
-      r.t_claim = ti.t_claim;
-      r.t_commit = t_commit;
-      r.slot = ti.slot;
-      r.tile = ti.tile;
-      r.cls = (int16_t)ti.cls;
-      r.kind = (int16_t)ti.kind;
-      r.cta = (int16_t)blockIdx.x;
-      unsigned smid;
-      asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
-      r.sm = (int16_t)smid;
-#ifdef MOE_LOG_ROWS
-      r.sm = (int16_t)ti.rows;
-#endif
-      a->log[idx] = r;
-    }
-  }
-}
-
-__device__ inline void build_queues(const RunArgs* a, SharedCtl* sc) {
-  sc->n_cls[0] = sc->n_cls[1] = 0;
-  sc->cum[0][0] = sc->cum[1][0] = 0;
-  for (int i = 0; i < a->n_ops; ++i) {
-    const int slot = a->slots[i];
-    const OpDev* op = &a->ops[slot];
-    const int cls = op->cls;
-    const int j = sc->n_cls[cls]++;
-    sc->cls_slot[cls][j] = slot;
-    sc->cls_free[cls][j] = (op->ready == nullptr && op->after_op < 0) ? 1 : 0;
-    sc->cum[cls][j + 1] = sc->cum[cls][j] + (unsigned)op_total_tiles(op, a->fuse_combine);
-  }
-}
-
-// silu(g) * u through the hardware tanh approximation (one special-function op per element;
-// its error, |g| * 2.4e-4 at worst, stays below the bf16 rounding of the result)
-__device__ __forceinline__ float silu_mul(float g, float u) {
-  float t;
-  asm("tanh.approx.f32 %0, %1;" : "=f"(t) : "f"(0.5f * g));
-  const float hg = 0.5f * g;
-  return fmaf(hg, t, hg) * u;                     // g * sigmoid(g) = g/2 * (1 + tanh(g/2))
-}
 
 // ------------------------------------------------------------------ FP8 (e4m3, fp32 block scales)
 // instruction descriptor: D fp32, A/B e4m3, both K-major, M = 128, N = 256
@@ -515,7 +246,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       mbar_init(&sc->iempty[s], 2 + kGatherThreads / 32);
       mbar_init(&sc->done[s], 256);
     }
-    build_queues(&args, sc);
+    build_queues(&args, &sc->qt);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_proxy();
   }
@@ -555,7 +286,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     ti.slot = ti.tile = ti.m = ti.row0 = ti.rows = ti.n = ti.kblocks = ti.expert = ti.cls = 0;
     ti.t_claim = 0;
     nx = ti;
-    claim_next(c, sc, rh, lane, ti, ti_need_ready);
+    claim_next(c, &sc->qt, rh, lane, ti, ti_need_ready);
     while (true) {
       ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);      // the claim loops exit warp-uniformly
       const OpDev* op = &args.ops[ti.kind == kEnd ? args.slots[0] : ti.slot];
@@ -609,7 +340,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           __syncwarp();
           if (++stage == kNS) { stage = 0; ph ^= 1u; }
           if (kb == claim_at)              // claim ahead (never blocks here)
-            have_nx = claim_once(c, sc, rh, lane, nx, nx_need_ready) == 1;
+            have_nx = claim_once(c, &sc->qt, rh, lane, nx, nx_need_ready) == 1;
           if (have_nx && !nx_published && kb > claim_at && kb >= ti.kblocks - kPublishLead) {
             // Hand the next tile to the other warps before this one's last loads go out, if that
             // takes no waiting: free ring slot, op ready, dependencies already met.
@@ -644,7 +375,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         ti_published = nx_published;
         have_nx = nx_published = false;
       } else {
-        claim_next(c, sc, rh, lane, ti, ti_need_ready);
+        claim_next(c, &sc->qt, rh, lane, ti, ti_need_ready);
       }
     }
   } else if (warp == 1) {

@@ -60,12 +60,13 @@ def test_decode_first_inside_the_budget_and_work_conserving():
     assert (outside["cls"] == 1).mean() > 0.9
     # work conserving: after the decode queue ran dry, budget CTAs went on with prefill tiles
     late = pre[pre["t_claim"] > t_dec_end]
-    assert len(np.unique(late["cta"][late["cta"] < q])) >= q // 2
-    assert len(np.unique(log["cta"])) == sm
+    units = sm // ctx.ctas_per_tile               # claiming units: CTAs, or pairs of CTAs
+    assert len(np.unique(late["cta"][late["cta"] < q])) >= q // ctx.ctas_per_tile // 2
+    assert len(np.unique(log["cta"])) == units
 
 
 def test_single_class_uses_all_ctas():
     ctx, log = _run(budget=16, n_ops=1)          # only the prefill op: decode budget must not idle CTAs
-    assert len(np.unique(log["cta"])) == ctx.sm_count
+    assert len(np.unique(log["cta"])) == ctx.sm_count // ctx.ctas_per_tile
     ctx, log = _run(budget=0, n_ops=2)           # budget 0: decode still gets served (by fallback)
     assert (log["cls"] == 0).sum() == ctx.footprint(1)[1]
