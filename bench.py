@@ -392,6 +392,7 @@ def run_ours(args):
     # ---- roofline of the dominant kernel (the persistent kernel), from live CUDA events
     launches = len(run_ms)
     t_run = float(np.mean(run_ms)) / 1e3
+    kernel_name = "moe_apk_pair_kernel" if w.ctx.ctas_per_tile == 2 else "moe_apk_kernel"
     flops_launch = w.flops / len(w.layers)
     bytes_launch = w.bytes_alg / len(w.layers)
     # the fp8 tensor peak is the measured bf16 peak x the nominal 2x ratio
@@ -404,7 +405,7 @@ def run_ours(args):
     else:
         roof = {"bound": "tensor", "achieved": flops_launch / t_run / 1e12,
                 "peak": tpeak, "unit": "TFLOP/s", "frac": tensor_frac}
-    roof.update({"traffic": None, "kernel": "moe_apk_kernel", "peak_source": peak_src,
+    roof.update({"traffic": None, "kernel": kernel_name, "peak_source": peak_src,
                  "launch_ms_mean": 1e3 * t_run, "launch_ms_min": float(np.min(run_ms)),
                  "algorithmic_flops_per_launch": flops_launch,
                  "algorithmic_bytes_per_launch": bytes_launch,

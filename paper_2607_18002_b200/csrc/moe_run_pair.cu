@@ -15,7 +15,7 @@
 // Roles per CTA (16 warps): leader only -- warp 0 scheduler (claims, waits for dependencies,
 // publishes tile descriptors to both CTAs), warp 1 MMA issuer, warp 2 committer; both CTAs --
 // warp 3 producer (TMA loads of its own half, read from the descriptor ring), warps 4-7 gather,
-// warps 8-15 epilogue.  Tile descriptors reach the second CTA through distributed shared
+// warps 8-15 epilogue; second CTA only -- warp 1 relays the completion of its gather to the leader.  Tile descriptors reach the second CTA through distributed shared
 // memory; its barrier arrivals that the leader waits for are remote mbarrier arrivals.  Every
 // wait is bounded, as in the single-CTA kernel.
 #include "moe_combine.cuh"
@@ -32,7 +32,7 @@ constexpr int kABytes = 128 * kRowBytes;                 // up to 128 activation
 constexpr int kBBytes = 128 * kRowBytes;                 // this CTA's 128 weight rows
 constexpr int kSB = kABytes + kBBytes;
 constexpr int kAccCols = 256;
-constexpr int kFullCount = 2 + 2 * (kGatherThreads / 32);
+constexpr int kFullCount = 2 + kGatherThreads + 1;
 // instruction descriptors: D fp32, A/B bf16, K-major, N = 256, M = 256 / 128 over the pair
 constexpr unsigned kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((256u >> 3) << 17);
 constexpr unsigned kIdesc256 = kIdescBase | ((256u >> 4) << 24);
@@ -41,10 +41,11 @@ constexpr unsigned kIdesc128 = kIdescBase | ((128u >> 4) << 24);
 struct SharedCtl {
   alignas(16) TileInfo info[kRing];
   // leader's: everything the MMAs of a stage read is in place.  kFullCount arrivals: one expect_tx
-  // per producer (TMA bytes of both CTAs) and one per gather warp of both CTAs (its rows have
-  // landed and are fenced for the tensor core); on tiles without a gather the leader's producer
-  // arrives in the gather warps' place
+  // per producer (TMA bytes of both CTAs), one per gather thread of the leader (completion of its
+  // cp.async copies) and one from the other CTA's relay warp (that CTA's gathered rows are in
+  // place); on tiles without a gather the leader's producer arrives in their place
   unsigned long long full[kNS];
+  unsigned long long fullA[kNS];     // second CTA: completion of its own gather threads' copies
   unsigned long long goA[kNS];       // producer -> gather warps: the stage may be overwritten
   unsigned long long empty[kNS];     // both (multicast commit): the stage's MMAs retired
   unsigned long long tfull[2];       // both (multicast commit): accumulator complete
@@ -178,7 +179,7 @@ __device__ __forceinline__ void issue_kblock(SharedCtl* sc, unsigned stages_addr
   // second weight box 64 rows (8 KB) on, second activation box 32 rows (4 KB) and 32 rows on
   static_assert(64 * kRowBytes == 8192 && 32 * kRowBytes == 4096, "offsets used by pair_issue_kblock");
   pair_issue_kblock(bar, p.tx, smem_u32(&sc->full[stage]),
-                    (leader && !p.g1) ? 2u * (kGatherThreads / 32) : 0u,   // nobody gathers for this tile
+                    (leader && !p.g1) ? (unsigned)kGatherThreads + 1u : 0u,   // nobody gathers for this tile
                     sB, p.tmw, kb * kBlockK, p.wy0, p.wy1, p.wy1 >= 0 ? 1u : 0u,
                     sA, p.tma, p.ay, (unsigned)p.a_boxes,
                     smem_u32(&sc->goA[stage]), p.g1 ? 1u : 0u);
@@ -212,6 +213,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
   if (threadIdx.x == 0) {
     for (int s = 0; s < kNS; ++s) {
       mbar_init(&sc->full[s], kFullCount);
+      mbar_init(&sc->fullA[s], kGatherThreads);
       mbar_init(&sc->goA[s], 1);
       mbar_init(&sc->empty[s], 1);
     }
@@ -220,10 +222,10 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       mbar_init(&sc->tempty[s], 16);
     }
     // a ring slot is released by: MMA warp, committer, producer, 4 gather warps (leader); producer,
-    // 4 gather warps (other CTA)
+    // relay, 4 gather warps (other CTA)
     for (int s = 0; s < kRing; ++s) {
       mbar_init(&sc->ifull[s], 1);
-      mbar_init(&sc->iempty[s], 12);
+      mbar_init(&sc->iempty[s], 13);
       mbar_init(&sc->done[s], 16);
       mbar_init(&sc->taken[s], 1);
     }
@@ -353,6 +355,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
         tc_fence_after();
         const unsigned d = __shfl_sync(0xffffffffu, tmem, 0) + b * (unsigned)kAccCols;
         const unsigned idesc = rows > kTileM ? kIdesc256 : kIdesc128;
+        const bool g1 = kind == kGateUp;
         bool fail = false;
         for (int kb = 0; kb < kblocks; ++kb) {
 #ifdef MOE_TIMING_PROBE
@@ -362,6 +365,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
 #ifdef MOE_TIMING_PROBE
           const long long q1 = clock64();
 #endif
+          if (g1) fence_async_proxy_smem();            // this CTA's cp.async-written rows -> tensor core reads
           const unsigned sA = sbase + stage * (unsigned)kSB;
           const unsigned long long ad = umma_desc(sA, kRowBytes), bd = umma_desc(sA + kABytes, kRowBytes);
 #pragma unroll
@@ -389,15 +393,42 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       args.dbg[49153] = clock64() - c_start;
     }
 #endif
+  } else if (warp == 1) {
+    // ============================================================ gather relay (second CTA)
+    // When this CTA's gather threads' copies of a stage have landed it makes them visible to the
+    // tensor core (proxy fence) and arrives on the leader's stage barrier.
+    int islot = 0;
+    unsigned iph = 0, kiter = 0, amask = 0;
+    while (true) {
+      if (!wait_info(c, &sc->ifull[islot], iph, 24, false)) break;
+      const int kind = sc->info[islot].kind;
+      const int kblocks = sc->info[islot].kblocks;
+      __syncwarp();
+      if (kind == kEnd) break;
+      if (lane == 0) arrive_at_leader(&sc->iempty[islot], false);
+      if (++islot == kRing) { islot = 0; iph ^= 1u; }
+      if (kind == kCombine) continue;
+      if (kind != kGateUp) { kiter += (unsigned)kblocks; continue; }
+      bool fail = false;
+      for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
+        const int stage = (int)(kiter % kNS);
+        if (!wwait(c, &sc->fullA[stage], (amask >> stage) & 1u, 25)) { fail = true; break; }
+        amask ^= 1u << stage;
+        if (lane == 0) {
+          fence_async_proxy_smem();
+          mbar_arrive_remote(map_to_cta(&sc->full[stage], 0));
+        }
+        __syncwarp();
+      }
+      if (fail) break;
+    }
   } else if (warp >= 4 && warp < 4 + kGatherThreads / 32) {
     // ============================================================ gather warps (cp.async)
     // This CTA's rows of a gate/up tile: row r of the tile is token sorted_to_flat[row0 + r] / k.
-    // A warp's copies of one k-block are one cp.async group; up to kLag + 1 groups are in flight.
-    // When the group issued kLag k-blocks earlier has landed the warp fences it for the tensor
-    // core and arrives once on the leader's stage barrier, so a warp never sits out the latency
-    // of its own copies.  Groups still in flight at the end of a tile are settled at once, oldest
-    // first -- after the token loads of the next tile have gone out when that tile is already
-    // published and gathers too.
+    // Eight adjacent lanes copy one 128-byte row slice.  Completion is asynchronous: every
+    // thread's copies arrive on a barrier when they land (the leader's stage barrier in the
+    // leader, a local one that the relay warp forwards in the other CTA), so these warps never
+    // wait for their own copies and run as far ahead of the MMAs as the producer does.
     const int gt = threadIdx.x - 128;
     constexpr int kCpr = kRowBytes / 16;                  // 16-byte chunks per row slice
     constexpr int kRowsPerPass = kGatherThreads / kCpr;   // 16 rows per cp.async round
@@ -405,33 +436,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
     const int chunk = gt % kCpr, rbase = gt / kCpr;
     int islot = 0;
     unsigned iph = 0, kiter = 0, gmask = 0;
-    // Stages whose arrival is still owed: the np stages before `nstage` (consecutive, modulo the
-    // ring), each with its cp.async group still outstanding, oldest first.
-    constexpr int kLag = 3;
-    int np = 0, nstage = 0;
-    auto settle_oldest = [&]() {                          // this warp's rows of the oldest owed stage have landed
-      const int st = (nstage - np + 2 * kNS) % kNS;
-      fence_async_proxy_smem();
-      __syncwarp();
-      if (lane == 0) {
-        if (leader) mbar_arrive(&sc->full[st]);
-        else mbar_arrive_remote(map_to_cta(&sc->full[st], 0));
-      }
-      --np;
-    };
-    auto drain = [&]() {                                  // oldest first, each as soon as it has landed
-      if (np >= 4) { cp_async_wait_group<3>(); settle_oldest(); }
-      if (np >= 3) { cp_async_wait_group<2>(); settle_oldest(); }
-      if (np >= 2) { cp_async_wait_group<1>(); settle_oldest(); }
-      if (np >= 1) { cp_async_wait_group<0>(); settle_oldest(); }
-    };
     while (true) {
-      if (np > 0) {
-        // drain now unless the next tile is there already and is a gate/up tile
-        const bool there = __all_sync(0xffffffffu, leader ? mbar_test(&sc->ifull[islot], iph)
-                                                           : mbar_try_cluster(&sc->ifull[islot], iph));
-        if (!there || sc->info[islot].kind != kGateUp) drain();
-      }
       if (!wait_info(c, &sc->ifull[islot], iph, 13, leader)) break;
       const int kind = sc->info[islot].kind;
       const int kblocks = sc->info[islot].kblocks;
@@ -449,13 +454,11 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       const int first = rank * rpc;                       // this CTA's first row of the tile
       int tok[kPasses];
 #pragma unroll
-      for (int j = 0; j < kPasses; ++j) {                 // the loads go out first ...
+      for (int j = 0; j < kPasses; ++j) {
         const int r = rbase + kRowsPerPass * j;
-        tok[j] = (r < rpc && first + r < rows) ? op->sorted_to_flat[row0 + first + r] : -1;
+        tok[j] = (r < rpc && first + r < rows) ? op->sorted_to_flat[row0 + first + r] / args.k : -1;
       }
-      drain();                                            // ... then what the previous tile still owes
-#pragma unroll
-      for (int j = 0; j < kPasses; ++j) tok[j] = tok[j] >= 0 ? tok[j] / args.k : -1;
+      unsigned long long* landed = leader ? sc->full : sc->fullA;
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
         const int stage = (int)(kiter % kNS);
@@ -469,17 +472,11 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
           if (tok[j] >= 0)     // the swizzle XORs the chunk index with the row's place in its 8-row group
             cp_async_16(sA + r * kRowBytes + ((chunk ^ (r & 7)) << 4), Xk + (size_t)tok[j] * pitch);
         }
-        cp_async_commit();
-        nstage = stage + 1 == kNS ? 0 : stage + 1;
-        ++np;
-        if (np > kLag) {
-          cp_async_wait_group<kLag>();                    // the group issued kLag k-blocks ago has landed
-          settle_oldest();
-        }
+        cp_async_arrive_noinc(&landed[stage]);
       }
       if (fail) break;
     }
-    drain();                                              // nothing stays armed, also after a failure
+    cp_async_wait_all();
   } else if (warp == 2 && leader) {
     // ============================================================ committer (leader)
     int islot = 0;
