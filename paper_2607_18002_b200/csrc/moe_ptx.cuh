@@ -339,4 +339,34 @@ __device__ __forceinline__ void pair_issue_kblock(unsigned bar, unsigned tx, uns
         "r"(go_bar), "r"(has_go)
       : "memory");
 }
+
+// One k-block of the pair's MMAs as ONE instruction group: the next stage's barrier is tested first and
+// the result is only read after the four MMAs and the commit have been issued, so that the barrier's
+// shared-memory round trip hides behind the issue of the MMAs.  Whole warp, warp-uniform operands; one
+// elected lane issues the MMAs and the commit.  Returns whether the next stage is already full.
+__device__ __forceinline__ bool pair_mma_kblock(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                                unsigned idesc, unsigned accumulate_first, unsigned empty_bar,
+                                                unsigned next_full_bar, unsigned next_parity) {
+  unsigned ready;
+  asm volatile(
+      "{\n\t.reg .pred e, p0, p1, pn;\n\t.reg .b32 r;\n\t.reg .b16 m;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "mov.b16 m, 3;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 pn, [%7], %8;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "setp.ne.b32 p0, %5, 0;\n\t"
+      "setp.eq.b32 p1, 0, 0;\n\t"
+      "add.u64 a1, %2, 2;\n\tadd.u64 a2, %2, 4;\n\tadd.u64 a3, %2, 6;\n\t"
+      "add.u64 b1, %3, 2;\n\tadd.u64 b2, %3, 4;\n\tadd.u64 b3, %3, 6;\n\t"
+      "@e tcgen05.mma.cta_group::2.kind::f16 [%1], %2, %3, %4, p0;\n\t"
+      "@e tcgen05.mma.cta_group::2.kind::f16 [%1], a1, b1, %4, p1;\n\t"
+      "@e tcgen05.mma.cta_group::2.kind::f16 [%1], a2, b2, %4, p1;\n\t"
+      "@e tcgen05.mma.cta_group::2.kind::f16 [%1], a3, b3, %4, p1;\n\t"
+      "@e tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%6], m;\n\t"
+      "selp.u32 %0, 1, 0, pn;\n\t}"
+      : "=r"(ready)
+      : "r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate_first), "r"(empty_bar),
+        "r"(next_full_bar), "r"(next_parity)
+      : "memory");
+  return ready != 0;
+}
 }  // namespace moe

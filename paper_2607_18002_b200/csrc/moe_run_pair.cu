@@ -357,28 +357,32 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
         const unsigned idesc = rows > kTileM ? kIdesc256 : kIdesc128;
         const bool g1 = kind == kGateUp;
         bool fail = false;
+        bool ready = false;                           // the current stage was seen full by the look-ahead test
+        const unsigned full0 = smem_u32(&sc->full[0]), empty0 = smem_u32(&sc->empty[0]);
         for (int kb = 0; kb < kblocks; ++kb) {
 #ifdef MOE_TIMING_PROBE
           const long long q0 = clock64();
 #endif
-          if (!wwait(c, &sc->full[stage], par, 8)) { fail = true; break; }
+          if (!ready && !wwait(c, &sc->full[stage], par, 8)) { fail = true; break; }
 #ifdef MOE_TIMING_PROBE
           const long long q1 = clock64();
 #endif
           if (g1) fence_async_proxy_smem();            // this CTA's cp.async-written rows -> tensor core reads
           const unsigned sA = sbase + stage * (unsigned)kSB;
           const unsigned long long ad = umma_desc(sA, kRowBytes), bd = umma_desc(sA + kABytes, kRowBytes);
-#pragma unroll
-          for (int k4 = 0; k4 < kBlockK / 16; ++k4)   // +32 bytes along K per step (>>4 = 2)
-            tc_mma2_bf16_elect(d, ad + 2ull * k4, bd + 2ull * k4, idesc, (kb | k4) ? 1u : 0u);
-          tc_commit_pair_elect(&sc->empty[stage]);    // frees the stage in both CTAs
+          const unsigned nstage = stage + 1 == kNS ? 0u : stage + 1, npar = stage + 1 == kNS ? par ^ 1u : par;
+          // four MMAs (+32 bytes along K per step: the descriptor's address field counts 16 bytes), the
+          // commit that frees the stage in both CTAs, and the test of the next stage's barrier
+          ready = pair_mma_kblock(d, ad, bd, idesc, kb ? 1u : 0u, empty0 + stage * 8u, full0 + nstage * 8u, npar);
+          ready = __all_sync(0xffffffffu, ready) && kb + 1 < kblocks;
 #ifdef MOE_TIMING_PROBE
           if (blockIdx.x == 14 && lane == 0 && dbg_i < 4096) {
             long long* pp = args.dbg + (size_t)dbg_i++ * 4;
             pp[0] = q0; pp[1] = q1; pp[2] = clock64(); pp[3] = kind * 100000 + rows * 100 + kb;
           }
 #endif
-          if (++stage == kNS) { stage = 0; par ^= 1u; }
+          stage = nstage;
+          par = npar;
         }
         if (fail) break;
         tc_commit_pair_elect(&sc->tfull[b]);            // accumulator complete, both CTAs
