@@ -137,6 +137,19 @@ int moe_combine(moe_ctx_t* ctx, int slot, void* stream);
  * the running kernel reads at every tile boundary.  0 <= decode_sms. */
 int moe_set_budget(moe_ctx_t* ctx, int decode_sms, void* stream);
 
+/* Online SM reallocation (Section 5.5, "Online SM Reallocation"): sets the budget word to
+ *     q' = min(q_max, ceil_c(q * x_moe / x_moe_star))
+ * where x_moe is the footprint of the decode op planned in `slot` (read on the device: the call
+ * is stream-ordered after that moe_plan and never synchronises), x_moe_star > 0 the footprint the
+ * static budget q was chosen for, and ceil_c rounds up to a multiple of c = moe_ctas_per_tile
+ * (the claiming unit: the paper's CTA cluster).  The product and quotient are taken in double
+ * precision.  MOE_ENOTPLANNED if the slot has no plan, MOE_EINVAL for q < 0, q_max < 0 or
+ * x_moe_star <= 0. */
+int moe_set_budget_scaled(moe_ctx_t* ctx, int slot, int q, double x_moe_star, int q_max, void* stream);
+
+/* Reads the budget word back (synchronous copy; call after synchronising the stream). */
+int moe_get_budget(moe_ctx_t* ctx, int32_t* out);
+
 /* Device status (synchronous copy; call after synchronising the stream).  code is 0 or
  * a MOE_E* value; detail[0..3] describe where (meaning depends on code).  Clears it. */
 int moe_status(moe_ctx_t* ctx, int32_t* code, int32_t detail[4]);

@@ -132,6 +132,15 @@ def plan(ids: np.ndarray, E: int):
     return counts, offsets, s2f, f2s
 
 
+def online_budget(q: int, x_moe: int, x_moe_star: float, q_max: int, c: int) -> int:
+    """Online SM reallocation (Section 5.5): q' = min(Q_max, ceil_c(q * x_moe / x_moe_star)), where ceil_c rounds
+    up to a multiple of the cluster size c."""
+    import math
+    want = math.ceil(q * x_moe / x_moe_star)
+    want = -(-want // c) * c
+    return min(q_max, want)
+
+
 def tiles(counts: np.ndarray, Mt: int):
     """-> (tile_expert, tile_row0, tile_rows); len == x_moe."""
     counts = np.ascontiguousarray(counts, dtype=np.int32)

@@ -27,7 +27,7 @@ MOE_CLASS_DECODE, MOE_CLASS_PREFILL = 0, 1
 MOE_TILE_M = 128
 
 EXPORTS = ("moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_run",
-           "moe_combine", "moe_set_budget", "moe_status", "moe_footprint",
+           "moe_combine", "moe_set_budget", "moe_set_budget_scaled", "moe_get_budget", "moe_status", "moe_footprint",
            "moe_read_tile_table", "moe_read_tile_log", "moe_sm_count", "moe_ctas_per_tile", "moe_strerror",
            "moe_plan_static")
 MOE_PLAN_STATIC_MAX_ROWS, MOE_PLAN_STATIC_MAX_EXPERTS = 32768, 256
@@ -89,6 +89,8 @@ def lib() -> C.CDLL:
         L.moe_run.argtypes = [vp, C.POINTER(i32), C.c_int, C.c_int, vp]
         L.moe_combine.argtypes = [vp, C.c_int, vp]
         L.moe_set_budget.argtypes = [vp, C.c_int, vp]
+        L.moe_set_budget_scaled.argtypes = [vp, C.c_int, C.c_int, C.c_double, C.c_int, vp]
+        L.moe_get_budget.argtypes = [vp, C.POINTER(i32)]
         L.moe_status.argtypes = [vp, C.POINTER(i32), C.POINTER(i32)]
         L.moe_footprint.argtypes = [vp, C.c_int, C.POINTER(i32), C.POINTER(i32)]
         L.moe_read_tile_table.argtypes = [vp, C.c_int, vp, C.c_int]
@@ -150,6 +152,17 @@ def moe_combine(ctx: int, slot: int, stream: int) -> None:
 def moe_set_budget(ctx: int, decode_sms: int, stream: int) -> None:
     _check(lib().moe_set_budget(C.c_void_p(ctx), int(decode_sms), C.c_void_p(stream)),
            "moe_set_budget")
+
+
+def moe_set_budget_scaled(ctx: int, slot: int, q: int, x_moe_star: float, q_max: int, stream: int) -> None:
+    _check(lib().moe_set_budget_scaled(C.c_void_p(ctx), int(slot), int(q), float(x_moe_star), int(q_max),
+                                       C.c_void_p(stream)), "moe_set_budget_scaled")
+
+
+def moe_get_budget(ctx: int) -> int:
+    out = C.c_int32()
+    _check(lib().moe_get_budget(C.c_void_p(ctx), C.byref(out)), "moe_get_budget")
+    return int(out.value)
 
 
 def moe_status(ctx: int):
@@ -294,6 +307,12 @@ class Context:
 
     def set_budget(self, decode_sms: int, stream=None):
         moe_set_budget(self.ctx, decode_sms, self._stream(stream))
+
+    def set_budget_scaled(self, slot: int, q: int, x_moe_star: float, q_max: int, stream=None):
+        moe_set_budget_scaled(self.ctx, slot, q, x_moe_star, q_max, self._stream(stream))
+
+    def get_budget(self) -> int:
+        return moe_get_budget(self.ctx)
 
     def status(self):
         return moe_status(self.ctx)

@@ -335,6 +335,30 @@ int moe_set_budget(moe_ctx_t* ctx, int decode_sms, void* stream) {
   return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ECUDA;
 }
 
+namespace {
+// q' = min(q_max, ceil_c(q * x_moe / x_star)) from the slot's planned footprint (Section 5.5)
+__global__ void scaled_budget_kernel(int* budget, const PlanState* plan, int q, double x_star, int q_max, int c) {
+  const double want = ceil((double)q * (double)plan->n_mtiles / x_star);
+  long long v = want > 2147483000.0 ? 2147483000ll : (long long)want;
+  v = (v + c - 1) / c * c;
+  *budget = (int)(v < (long long)q_max ? v : (long long)q_max);
+}
+}  // namespace
+
+int moe_set_budget_scaled(moe_ctx_t* ctx, int slot, int q, double x_moe_star, int q_max, void* stream) {
+  if (!ctx || slot < 0 || slot >= ctx->cfg.max_ops || q < 0 || q_max < 0 || !(x_moe_star > 0.0)) return MOE_EINVAL;
+  if (!ctx->planned[slot]) return MOE_ENOTPLANNED;
+  const PlanState* ps = reinterpret_cast<const PlanState*>(ctx->slot_base(slot) + ctx->L.plan_off);
+  scaled_budget_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(&ctx->g()->budget, ps, q, x_moe_star, q_max,
+                                                                      ctx->pair_kernel ? 2 : 1);
+  return cudaGetLastError() == cudaSuccess ? MOE_OK : MOE_ECUDA;
+}
+
+int moe_get_budget(moe_ctx_t* ctx, int32_t* out) {
+  if (!ctx || !out) return MOE_EINVAL;
+  return cudaMemcpy(out, &ctx->g()->budget, sizeof(int32_t), cudaMemcpyDeviceToHost) == cudaSuccess ? MOE_OK : MOE_ECUDA;
+}
+
 int moe_status(moe_ctx_t* ctx, int32_t* code, int32_t detail[4]) {
   if (!ctx || !code) return MOE_EINVAL;
   Status s;

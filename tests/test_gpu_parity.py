@@ -149,7 +149,8 @@ def test_one_expert_takes_everything_and_empty_op():
 
 def test_schedule_independence_bitwise():
     """A phase switch happens only between tiles, so the output may not depend on the budget,
-    on the class split, on fusing the combine, or on the run."""
+    on the class split, on fusing the combine, on the grid (and with it on the kernel: CTA
+    pairs or single CTAs), or on the run."""
     spec = SMALL
     W = synth.make_weights(spec)
     ops = synth.make_ops(spec)
@@ -157,6 +158,9 @@ def test_schedule_independence_bitwise():
     for fuse, budget, n_ctas in ((False, 0, 0), (True, 0, 0), (True, 16, 0), (True, 1000, 0),
                                  (True, 64, 3), (True, 1, 1), (True, 0, 0)):
         ctx, bound, _, _ = _run_spec(spec, fuse, budget=budget, ops=ops, W=W, n_ctas=n_ctas)
+        # an even grid runs bf16 on CTA pairs (one MMA over two SMs), an odd one on single CTAs:
+        # the comparison below therefore also holds the two kernels to the same bits
+        assert ctx.ctas_per_tile == (1 if n_ctas % 2 else 2)
         outs.append([b.y.clone() for b in bound])
     for o in outs[1:]:
         for a, b in zip(outs[0], o):

@@ -70,3 +70,18 @@ def test_single_class_uses_all_ctas():
     assert len(np.unique(log["cta"])) == ctx.sm_count // ctx.ctas_per_tile
     ctx, log = _run(budget=0, n_ops=2)           # budget 0: decode still gets served (by fallback)
     assert (log["cls"] == 0).sum() == ctx.footprint(1)[1]
+
+
+def test_scaled_budget_matches_the_formula():
+    """moe_set_budget_scaled computes q' of Section 5.5 on the device from the planned footprint."""
+    import oracle
+    ctx, log = _run(budget=16, n_ops=2)
+    x_dec = ctx.footprint(1)[0]                       # slot 1 is the decode op
+    c = ctx.ctas_per_tile
+    for q, x_star, q_max in ((32, float(x_dec), 148), (32, x_dec / 2.0, 148), (32, x_dec / 7.0, 96),
+                             (5, x_dec * 1.5, 148), (0, 10.0, 148), (33, x_dec - 0.5, 148)):
+        ctx.set_budget_scaled(1, q, x_star, q_max)
+        torch.cuda.synchronize()
+        assert ctx.get_budget() == oracle.online_budget(q, x_dec, x_star, q_max, c), (q, x_star, q_max)
+    with pytest.raises(moe.MoeError):
+        ctx.set_budget_scaled(1, 32, 0.0, 148)

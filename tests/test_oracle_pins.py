@@ -298,3 +298,25 @@ def test_fp8_path_equals_dense_on_dequantised_inputs():
     out_q = oracle.forward(W, op.x, op.x_scale, op.ids, op.w, round_A=oracle.ROUND_E4M3_1X128)
     rel = np.linalg.norm(out_q["y"] - out["y"]) / np.linalg.norm(out["y"])
     assert 1e-3 < rel < 6e-2
+
+
+def test_online_budget_closed_forms_and_brute_force():
+    """Section 5.5: q' = min(Q_max, ceil_c(q x_moe / x_moe*)).  Closed forms, and exact rational arithmetic
+    on a grid (a wrong rounding direction, a forgotten cap or a forgotten cluster multiple fails one)."""
+    from fractions import Fraction
+    ob = oracle.online_budget
+    assert ob(32, 100, 100, 148, 1) == 32            # footprint as expected: the static budget
+    assert ob(32, 200, 100, 148, 1) == 64            # twice the footprint: twice the budget
+    assert ob(32, 1000, 100, 96, 1) == 96            # capped: Q_max preserves prefill progress
+    assert ob(32, 0, 100, 148, 2) == 0               # nothing to run
+    assert ob(3, 100, 100, 148, 2) == 4              # rounded UP to a cluster multiple
+    assert ob(32, 101, 100, 148, 1) == 33            # ceil, not round
+    for q in (0, 1, 7, 32, 64):
+        for x in (0, 1, 5, 99, 100, 101, 250):
+            for xs in (1, 3, 100, 128):
+                for c in (1, 2, 4):
+                    exact = Fraction(q * x, xs)
+                    ceil = -((-exact.numerator) // exact.denominator)
+                    ceil_c = -(-ceil // c) * c
+                    assert ob(q, x, xs, 120, c) == min(120, ceil_c)
+                    assert ob(q, x, xs, 120, c) % c == 0 or ob(q, x, xs, 120, c) == 120
