@@ -9,7 +9,7 @@
  *
  * (the paper's Section 2.1 MoE module; the kernel that runs it is the adaptive
  * persistent kernel of Section 4: two grouped GEMMs, the activation, the MoE pre- and
- * post-processing and the tile scheduler in one launch, Section 6.1).
+ * post-processing and the tile scheduler in one launch, Section 7.1).
  *
  * Conventions
  *   - Every pointer in moe_op_t and the workspace is a DEVICE pointer owned by the
@@ -49,7 +49,7 @@ enum {
 enum { MOE_DTYPE_BF16 = 0, MOE_DTYPE_FP8_E4M3 = 1 };
 enum { MOE_CLASS_DECODE = 0, MOE_CLASS_PREFILL = 1 };
 
-/* Height of a token-dimension tile (the M_t of the footprint formula, Section 5.2). */
+/* Height of a token-dimension tile (the M_t of the footprint formula, Section 6.2). */
 #define MOE_TILE_M 128
 
 typedef struct moe_ctx moe_ctx_t; /* opaque, host side */
@@ -61,7 +61,7 @@ typedef struct {
   int32_t inter;             /* I, multiple of 128                                       */
   int32_t dtype;             /* MOE_DTYPE_*                                              */
   int32_t max_tokens_per_op; /* sizes the per-slot scratch; buffers are fixed up front,  */
-  int32_t max_ops;           /* as the paper's preallocated final buffers (Section 4.4)  */
+  int32_t max_ops;           /* as the paper's preallocated final buffers (Section 5.2)  */
   int32_t wait_limit_us;     /* device-side wait budget before MOE_ETIMEOUT; 0 = 2 s     */
   int32_t tile_log_entries;  /* capacity of the per-tile log; 0 = logging off            */
   int32_t n_ctas;            /* persistent grid size; 0 = one CTA per SM                 */
@@ -89,7 +89,7 @@ typedef struct {
 } moe_op_t;
 
 /* One record per executed tile (only when tile_log_entries > 0). Times are GPU
- * globaltimer nanoseconds; the preemption-interval analysis of Section 6.5 is made
+ * globaltimer nanoseconds; the preemption-interval analysis of Section 7.6 is made
  * from these. */
 typedef struct {
   uint64_t t_claim;  /* the tile was taken from its queue                                 */
@@ -111,8 +111,8 @@ void moe_destroy(moe_ctx_t* ctx);
 
 /* Plan (pre-processing): top-k ids -> counts, exclusive offsets by a device prefix
  * sum, the stable permutation (rows of an expert keep ascending flat index -- the
- * packed per-expert layout of Section 2.3), and the op's tile table, whose length is
- * the footprint x_moe = sum_{e: m_e>0} ceil(m_e / M_t) of Section 5.2.  Binds `op` to
+ * packed per-expert layout of Section 2.4), and the op's tile table, whose length is
+ * the footprint x_moe = sum_{e: m_e>0} ceil(m_e / M_t) of Section 6.2.  Binds `op` to
  * `slot`; the struct is copied, the buffers it names must stay valid until the work
  * enqueued on them has finished. */
 int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
@@ -121,7 +121,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
  * repeatedly claims the next tile from the decode queue or the prefill queue of
  * Section 4.2 -- CTAs with index below the decode budget prefer decode tiles, the
  * others prefill tiles, each falling back to the other class when its own has nothing
- * ready (Section 5.4) -- and runs it: gate/up grouped GEMM with fused SwiGLU, then the
+ * ready (Section 6.4) -- and runs it: gate/up grouped GEMM with fused SwiGLU, then the
  * down grouped GEMM, on rows gathered through the permutation.  A phase switch happens
  * only between tiles (Section 4.2), so results do not depend on the schedule.
  * Ops of one class are served in the order given.  With fuse_combine != 0 the
@@ -133,11 +133,11 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
  * order j = 0..k-1 in fp32 (Section 2.1, "combines their outputs"). */
 int moe_combine(moe_ctx_t* ctx, int slot, void* stream);
 
-/* Decode SM budget q of Section 5.4: a stream-ordered 4-byte write to the device word
+/* Decode SM budget q of Section 6.4: a stream-ordered 4-byte write to the device word
  * the running kernel reads at every tile boundary.  0 <= decode_sms. */
 int moe_set_budget(moe_ctx_t* ctx, int decode_sms, void* stream);
 
-/* Online SM reallocation (Section 5.5, "Online SM Reallocation"): sets the budget word to
+/* Online SM reallocation (Section 6.4, "Online SM Reallocation"): sets the budget word to
  *     q' = min(q_max, ceil_c(q * x_moe / x_moe_star))
  * where x_moe is the footprint of the decode op planned in `slot` (read on the device: the call
  * is stream-ordered after that moe_plan and never synchronises), x_moe_star > 0 the footprint the

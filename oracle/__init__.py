@@ -133,7 +133,7 @@ def plan(ids: np.ndarray, E: int):
 
 
 def online_budget(q: int, x_moe: int, x_moe_star: float, q_max: int, c: int) -> int:
-    """Online SM reallocation (Section 5.5): q' = min(Q_max, ceil_c(q * x_moe / x_moe_star)), where ceil_c rounds
+    """Online SM reallocation (Section 6.4): q' = min(Q_max, ceil_c(q * x_moe / x_moe_star)), where ceil_c rounds
     up to a multiple of the cluster size c."""
     import math
     want = math.ceil(q * x_moe / x_moe_star)

@@ -9,10 +9,10 @@
  * definition written out, step by step, with double accumulators:
  *
  *   plan     counts / exclusive offsets / stable permutation of the routed rows
- *            (the per-expert packed layout of Section 2.3) and the tile table
- *            whose length is the footprint x_moe of Section 5.2
+ *            (the per-expert packed layout of Section 2.4) and the tile table
+ *            whose length is the footprint x_moe of Section 6.2
  *   ffn      per routed row, SwiGLU expert FFN: silu(x Wg) * (x Wu), then Wd
- *            (the "two grouped GEMMs, activation functions" of Section 6.1)
+ *            (the "two grouped GEMMs, activation functions" of Section 7.1)
  *   combine  y[t] = sum_j w[t,j] * d[row(t,j)], slots in order
  *
  * Parity pins (see tests/test_oracle_pins.py): the plan equals a stable argsort
@@ -165,7 +165,7 @@ int orc_plan(const int32_t* ids, int R, int E, int32_t* counts, int32_t* offsets
 }
 
 /* Tile table: for every expert with rows, ceil(m_e / M_t) tiles of (expert, first
- * sorted row, valid rows).  The return value is x_moe (Section 5.2).  Output
+ * sorted row, valid rows).  The return value is x_moe (Section 6.2).  Output
  * arrays may be NULL to only count. */
 int orc_tiles(const int32_t* counts, int E, int Mt, int32_t* t_expert, int32_t* t_row0,
               int32_t* t_rows) {

@@ -102,7 +102,7 @@ struct Status {   // first error wins (atomicCAS on code)
 
 struct Global {
   Status status;
-  int budget;             // decode SM budget q (Section 5.4)
+  int budget;             // decode SM budget q (Section 6.4)
   int pad[7];
 };
 

@@ -336,7 +336,7 @@ int moe_set_budget(moe_ctx_t* ctx, int decode_sms, void* stream) {
 }
 
 namespace {
-// q' = min(q_max, ceil_c(q * x_moe / x_star)) from the slot's planned footprint (Section 5.5)
+// q' = min(q_max, ceil_c(q * x_moe / x_star)) from the slot's planned footprint (Section 6.4)
 __global__ void scaled_budget_kernel(int* budget, const PlanState* plan, int q, double x_star, int q_max, int c) {
   const double want = ceil((double)q * (double)plan->n_mtiles / x_star);
   long long v = want > 2147483000.0 ? 2147483000ll : (long long)want;

@@ -1,6 +1,6 @@
 // moe_plan: top-k expert ids -> per-expert counts, exclusive offsets (device prefix sum),
 // the stable permutation of routed rows, the m-tile table (its length is the footprint
-// x_moe of Section 5.2 of the paper) and the ordered tile list the persistent kernel's
+// x_moe of Section 6.2 of the paper) and the ordered tile list the persistent kernel's
 // queues serve.
 //
 // The permutation is one stable counting-sort pass over the expert id.  No atomic decides

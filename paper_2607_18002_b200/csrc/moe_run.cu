@@ -5,7 +5,7 @@
 //   warp 0      scheduler + producer.  At every tile boundary it reads the decode budget
 //               word and the two queue heads, claims the next tile (decode first for CTAs
 //               below the budget, prefill first for the others, each falling back to the
-//               other class: Sections 4.2 and 5.4), hands the tile to the other warps
+//               other class: Sections 4.2 and 6.4), hands the tile to the other warps
 //               through a shared-memory ring guarded by mbarriers (the hand-off of
 //               Section 4.3: the first pipeline warp decides, later warps follow), waits for
 //               the tile's dependencies, then feeds the pipeline: weight tiles (and the

@@ -1,7 +1,7 @@
 // moe_run on CTA pairs: the bf16 persistent expert kernel with two SMs per tile.
 //
 // Same scheduling as the single-CTA kernel (two queues, budget word, claim at tile
-// boundaries: Sections 4.2 and 5.4), but the unit that claims and runs a tile is a cluster of
+// boundaries: Sections 4.2 and 6.4), but the unit that claims and runs a tile is a cluster of
 // two CTAs on neighbouring SMs, and the MMAs are tcgen05.mma.cta_group::2:
 //   - a tile of up to 256 rows runs as ONE M = 256 instruction per k-step: each CTA holds 128
 //     of its rows (activations) and 128 of the 256 weight rows of the tile in its own shared

@@ -1,5 +1,5 @@
 // Scheduling pieces shared by the persistent kernels: bounded waits, the two-class tile queue
-// (Sections 4.2 and 5.4), tile publication and the SwiGLU helper.
+// (Sections 4.2 and 6.4), tile publication and the SwiGLU helper.
 #pragma once
 #include "moe_dev.cuh"
 #include "moe_ptx.cuh"

@@ -73,7 +73,7 @@ def test_single_class_uses_all_ctas():
 
 
 def test_scaled_budget_matches_the_formula():
-    """moe_set_budget_scaled computes q' of Section 5.5 on the device from the planned footprint."""
+    """moe_set_budget_scaled computes q' of Section 6.4 on the device from the planned footprint."""
     import oracle
     ctx, log = _run(budget=16, n_ops=2)
     x_dec = ctx.footprint(1)[0]                       # slot 1 is the decode op

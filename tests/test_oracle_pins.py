@@ -79,7 +79,7 @@ def test_tiles_closed_form(Mt):
     counts[[3, 10]] = 0
     counts[5], counts[6], counts[7] = Mt, Mt + 1, Mt - 1
     te, t0, tr = oracle.tiles(counts, Mt)
-    x_moe = sum(-(-int(c) // Mt) for c in counts if c > 0)        # Section 5.2 footprint
+    x_moe = sum(-(-int(c) // Mt) for c in counts if c > 0)        # Section 6.2 footprint
     assert len(te) == x_moe
     assert tr.sum() == counts.sum() and tr.min() >= 1 and tr.max() <= Mt
     offsets = np.concatenate([[0], np.cumsum(counts)])
@@ -301,7 +301,7 @@ def test_fp8_path_equals_dense_on_dequantised_inputs():
 
 
 def test_online_budget_closed_forms_and_brute_force():
-    """Section 5.5: q' = min(Q_max, ceil_c(q x_moe / x_moe*)).  Closed forms, and exact rational arithmetic
+    """Section 6.4: q' = min(Q_max, ceil_c(q x_moe / x_moe*)).  Closed forms, and exact rational arithmetic
     on a grid (a wrong rounding direction, a forgotten cap or a forgotten cluster multiple fails one)."""
     from fractions import Fraction
     ob = oracle.online_budget

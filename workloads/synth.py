@@ -7,8 +7,8 @@ CPU oracle and the CUDA library consume the same bytes.  It imports neither of
 them.
 
 Workloads (shapes follow the paper's evaluation setting of 256 routed experts
-with top-8 routing, Section 6.1, and a decode batch of 128 tokens next to a
-prefill batch of 8192 tokens, Section 6.3):
+with top-8 routing, Section 7.1, and a decode batch of 128 tokens next to a
+prefill batch of 8192 tokens, Section 7.3):
 
   c1  tiny bf16 layer, 48 prefill + 16 decode tokens, softmax -> top-2 router
   c2  decode-only bf16 layer, 128 tokens, uniform top-8 of 256
