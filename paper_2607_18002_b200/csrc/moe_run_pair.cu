@@ -274,6 +274,9 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
       ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);
+      // The gather warps will read the tile's row list (4 bytes per row) first thing: pull it into L2
+      // now, the weight stream has usually pushed it out since the plan wrote it.
+      if (ti.kind == kGateUp && lane * 32 < ti.rows) prefetch_l2(op->sorted_to_flat + ti.row0 + lane * 32);
       if (ti.kind == kEnd || !ok) break;
       if (!wwait(c, &sc->taken[islot], iph, 26)) break;
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
