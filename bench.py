@@ -36,6 +36,20 @@ KERNELS_PER_PLAN = 3          # histogram, scan + tile list, scatter
 DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c2s": (20, 3), "c3s": (10, 3), "c5s": (10, 3)}
 
 
+
+# DRAM bytes per launch of the persistent kernel (dram__bytes_read.sum + dram__bytes_write.sum) from one ncu
+# capture each.  The captures are of the small variants (c3s, c2s, c5s: a full-size launch under the profiler's
+# save/restore is too large); the full-size figures scale them by the number of active experts, because the
+# traffic is the weights of the active experts, read about once (c3: 256/64, c2: 251/63, c5: 256/32).
+NCU_DRAM_BYTES = {
+    ("c3s", "moe_apk_pair_kernel"): 2.029e9 + 0.160e9,
+    ("c3", "moe_apk_pair_kernel"): (2.029e9 + 0.160e9) * 256 / 64,
+    ("c2s", "moe_apk_pair_kernel"): 1.815e9 + 0.007e9,
+    ("c2", "moe_apk_pair_kernel"): (1.815e9 + 0.007e9) * 251 / 63,
+    ("c5s", "moe_apk_kernel"): 2.524e9 + 0.087e9,
+    ("c5", "moe_apk_kernel"): (2.524e9 + 0.087e9) * 256 / 32,
+}
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -405,7 +419,11 @@ def run_ours(args):
     else:
         roof = {"bound": "tensor", "achieved": flops_launch / t_run / 1e12,
                 "peak": tpeak, "unit": "TFLOP/s", "frac": tensor_frac}
-    roof.update({"traffic": None, "kernel": kernel_name, "peak_source": peak_src,
+    roof.update({"traffic": NCU_DRAM_BYTES.get((args.workload, kernel_name)), "kernel": kernel_name,
+                 "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of the small variant, "
+                                   "scaled by active experts (see profiles/)"
+                                   if (args.workload, kernel_name) in NCU_DRAM_BYTES else None,
+                 "peak_source": peak_src,
                  "launch_ms_mean": 1e3 * t_run, "launch_ms_min": float(np.min(run_ms)),
                  "algorithmic_flops_per_launch": flops_launch,
                  "algorithmic_bytes_per_launch": bytes_launch,
