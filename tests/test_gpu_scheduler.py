@@ -85,3 +85,16 @@ def test_scaled_budget_matches_the_formula():
         assert ctx.get_budget() == oracle.online_budget(q, x_dec, x_star, q_max, c), (q, x_star, q_max)
     with pytest.raises(moe.MoeError):
         ctx.set_budget_scaled(1, 32, 0.0, 148)
+
+
+def test_latency_follows_the_footprint_not_the_token_count():
+    """Section 6.2: at a fixed token count the kernel time grows with the number of active experts
+    (x_moe), and an affine law in x_moe describes it; a small shape keeps this quick."""
+    from paper_2607_18002_b200.latency_model import fit_affine, sweep
+    rows = sweep(E=64, k=4, H=1024, I=512, tokens=(16, 64), actives=(4, 16, 64), reps=6)
+    for T in (16, 64):
+        us = [r["us"] for r in rows if r["tokens"] == T]
+        assert us[0] < us[-1]                                  # more active experts, same tokens: slower
+    assert all(r["x_moe"] == r["active"] for r in rows)        # every active expert holds < 128 rows: one tile each
+    alpha, beta, r2 = fit_affine([r["x_moe"] for r in rows], [r["us"] for r in rows])
+    assert beta > 0 and r2 > 0.8

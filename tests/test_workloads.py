@@ -1,4 +1,5 @@
 """The seeded input generator: determinism, routing validity and the stated shapes."""
+import pytest
 import numpy as np
 import torch
 
@@ -53,3 +54,23 @@ def test_tensors_deterministic_and_fp8_blocks():
     c1 = synth.make_weights(synth.SPECS["c1"], threads=1)
     assert c1.w_gate_up.dtype == torch.bfloat16 and c1.w_gate_up.shape == (8, 1024, 256)
     assert abs(c1.w_gate_up.float().std().item() - 0.02) < 1e-3
+
+
+def test_route_active_pool_uses_exactly_the_pool():
+    rng = np.random.default_rng(3)
+    ids, w = synth.route_active_pool(rng, 64, 4, 32, 8)
+    assert ids.shape == (64, 4) and len(np.unique(ids)) == 8
+    assert all(len(set(r)) == 4 for r in ids.tolist())
+    assert np.allclose(w.sum(axis=1), 1.0, atol=1e-6)
+    with pytest.raises(ValueError):
+        synth.route_active_pool(rng, 4, 4, 32, 2)
+
+
+def test_latency_model_fit_recovers_an_affine_law():
+    from paper_2607_18002_b200.latency_model import fit_affine
+    x = np.array([8, 16, 32, 64, 128, 256], dtype=np.float64)
+    a, b, r2 = fit_affine(x, 40.0 + 4.5 * x)
+    assert abs(a - 40.0) < 1e-9 and abs(b - 4.5) < 1e-9 and r2 > 1 - 1e-12
+    rng = np.random.default_rng(0)
+    a, b, r2 = fit_affine(x, 40.0 + 4.5 * x + rng.normal(0, 1.0, x.shape))
+    assert abs(b - 4.5) < 0.1 and r2 > 0.99

@@ -220,6 +220,21 @@ def route_popularity(rng, T: int, k: int, log_pi: np.ndarray):
     return _weights_over_chosen(rng, ids)
 
 
+def route_active_pool(rng, T: int, k: int, E: int, n_active: int):
+    """k distinct experts per token, uniform over a seeded pool of `n_active` of the E experts:
+    the same number of tokens with a chosen number of active experts (the setting of the paper's
+    tile-aware latency model, Section 6.2)."""
+    if not k <= n_active <= E:
+        raise ValueError("need k <= n_active <= E")
+    pool = np.sort(rng.permutation(E)[:n_active])
+    log_pi = np.full(E, -np.inf)
+    log_pi[pool] = 0.0
+    g = rng.gumbel(size=(T, E))
+    keys = np.where(np.isfinite(log_pi)[None, :], g, -np.inf)
+    ids = np.argpartition(-keys, k - 1, axis=1)[:, :k].astype(np.int32)
+    return _weights_over_chosen(rng, ids)
+
+
 def zipf_log_pi(rng, E: int, s: float) -> np.ndarray:
     rank = rng.permutation(E) + 1           # seeded random expert order
     return -s * np.log(rank.astype(np.float64))
