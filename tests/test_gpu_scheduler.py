@@ -98,3 +98,15 @@ def test_latency_follows_the_footprint_not_the_token_count():
     assert all(r["x_moe"] == r["active"] for r in rows)        # every active expert holds < 128 rows: one tile each
     alpha, beta, r2 = fit_affine([r["x_moe"] for r in rows], [r["us"] for r in rows])
     assert beta > 0 and r2 > 0.8
+
+
+def test_sharing_study_runs_and_launch_granularity_sharing_serialises():
+    """Two whole-grid launches cannot overlap (one CTA per SM): the decode launch on the high-priority
+    stream still ends after the prefill launch, while one persistent launch with a large decode budget
+    finishes the decode operation well before the prefill operation (Section 7.3's comparison, small shape)."""
+    from paper_2607_18002_b200.sharing_study import study
+    rows = study(E=32, k=4, H=1024, I=512, prefill_tokens=8192, decode_tokens=64, budgets=(96,), reps=3)
+    by = {(r["arm"], r["q"]): r for r in rows}
+    assert all(r["prefill_us"] > 0 and r["decode_us"] > 0 for r in rows)
+    assert by[("streams", None)]["decode_us"] > by[("exclusive", None)]["prefill_us"] * 0.9
+    assert by[("apk", 96)]["decode_us"] < by[("apk", 96)]["prefill_us"]
