@@ -1,5 +1,6 @@
 // moe_run: the persistent expert kernel (the adaptive persistent kernel of Section 4 of the
-// paper, rebuilt for sm_100a).
+// paper, rebuilt for sm_100a), one CTA per tile.  This kernel runs the FP8 e4m3 path, and bf16 on
+// grids with an odd number of CTAs; bf16 on an even grid runs on CTA pairs (moe_run_pair.cu).
 //
 // One CTA per SM, 16 warps with fixed roles:
 //   warp 0      scheduler + producer.  At every tile boundary it reads the decode budget

@@ -251,9 +251,6 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
       unsigned smid;
       asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
       r.sm = (int16_t)smid;
-#ifdef MOE_LOG_ROWS
-      r.sm = (int16_t)ti.rows;
-#endif
       a->log[idx] = r;
     }
   }
