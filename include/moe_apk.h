@@ -189,6 +189,15 @@ int moe_plan_static(const int32_t* topk_ids, int32_t n_tokens, int32_t top_k, in
                     int32_t* counts, int32_t* offsets, int32_t* sorted_to_flat,
                     int32_t* flat_to_sorted, void* stream);
 
+/* The router ahead of moe_plan (Section 2.1: a router selects the top-k routed experts of each
+ * token; the arithmetic is this library's reading -- softmax over the experts, the k largest,
+ * weights renormalised over those k).  logits [T, E] fp32 -> topk_ids [T, k] (in order of
+ * decreasing logit, ties to the lower expert id) and topk_w [T, k] fp32 (they sum to 1).  All
+ * pointers are device pointers; no context, no workspace.  n_experts <= 1024, top_k <= 32 and
+ * <= n_experts, else MOE_EINVAL.  Logits must be finite. */
+int moe_route(const float* logits, int32_t n_tokens, int32_t n_experts, int32_t top_k,
+              int32_t* topk_ids, float* topk_w, void* stream);
+
 /* Multiprocessor count of the context's device (the default persistent grid). */
 int moe_sm_count(moe_ctx_t* ctx);
 

@@ -29,7 +29,7 @@ MOE_TILE_M = 128
 EXPORTS = ("moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_run",
            "moe_combine", "moe_set_budget", "moe_set_budget_scaled", "moe_get_budget", "moe_status", "moe_footprint",
            "moe_read_tile_table", "moe_read_tile_log", "moe_sm_count", "moe_ctas_per_tile", "moe_strerror",
-           "moe_plan_static")
+           "moe_plan_static", "moe_route")
 MOE_PLAN_STATIC_MAX_ROWS, MOE_PLAN_STATIC_MAX_EXPERTS = 32768, 256
 
 
@@ -96,6 +96,7 @@ def lib() -> C.CDLL:
         L.moe_read_tile_table.argtypes = [vp, C.c_int, vp, C.c_int]
         L.moe_read_tile_log.argtypes = [vp, vp, C.c_int, C.POINTER(C.c_int)]
         L.moe_plan_static.argtypes = [vp, i32, i32, i32, vp, vp, vp, vp, vp]
+        L.moe_route.argtypes = [vp, i32, i32, i32, vp, vp, vp]
         L.moe_sm_count.argtypes = [vp]
         L.moe_ctas_per_tile.argtypes = [vp]
         L.moe_strerror.argtypes = [C.c_int]
@@ -203,6 +204,25 @@ def moe_plan_static(topk_ids_ptr: int, n_tokens: int, top_k: int, n_experts: int
                                  C.c_void_p(counts_ptr), C.c_void_p(offsets_ptr),
                                  C.c_void_p(sorted_to_flat_ptr), C.c_void_p(flat_to_sorted_ptr),
                                  C.c_void_p(stream)), "moe_plan_static")
+
+
+def moe_route(logits_ptr: int, n_tokens: int, n_experts: int, top_k: int, ids_ptr: int, w_ptr: int,
+              stream: int) -> None:
+    _check(lib().moe_route(C.c_void_p(logits_ptr), int(n_tokens), int(n_experts), int(top_k),
+                           C.c_void_p(ids_ptr), C.c_void_p(w_ptr), C.c_void_p(stream)), "moe_route")
+
+
+def route(logits, top_k: int, stream=None):
+    """logits: CUDA fp32 tensor [T, E] -> (topk_ids int32 [T, k], topk_w fp32 [T, k])."""
+    import torch
+    if not (logits.is_cuda and logits.dtype == torch.float32 and logits.dim() == 2 and logits.is_contiguous()):
+        raise ValueError("logits must be a contiguous CUDA fp32 [T, E] tensor")
+    T, E = logits.shape
+    ids = torch.empty((T, top_k), dtype=torch.int32, device=logits.device)
+    w = torch.empty((T, top_k), dtype=torch.float32, device=logits.device)
+    s = torch.cuda.current_stream(logits.device) if stream is None else stream
+    moe_route(logits.data_ptr(), T, E, top_k, ids.data_ptr(), w.data_ptr(), int(s.cuda_stream))
+    return ids, w
 
 
 def moe_sm_count(ctx: int) -> int:
