@@ -198,24 +198,68 @@ class Workload:
                 e1.record()
                 ev.append((e0, e1))
 
-    def step_e2e(self):
-        """The same step with host buffers: inputs come from pinned host memory and the
-        result goes back to it, all inside the timed region."""
-        ctx = self.ctx
-        for li, (_, bound, host) in enumerate(self.layers):
-            if self.spec.layers > 1:
-                ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
-            for s, (b, (hx, hi, hw, hy, hs)) in enumerate(zip(bound, host)):
-                b.x.copy_(hx, non_blocking=True)
-                if hs is not None:
-                    b.x_scale.copy_(hs, non_blocking=True)
-                b.topk_ids.copy_(hi, non_blocking=True)
-                b.topk_w.copy_(hw, non_blocking=True)
-                ctx.plan(s, b)
-            ctx.run(list(range(len(bound))), fuse_combine=True)
-            for b, (_, _, _, hy, _) in zip(bound, host):
-                hy.copy_(b.y, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+    def _second_set(self):
+        """A second context and a second set of device buffers for every op: the end-to-end loop
+        alternates between the two sets, so that the copies of one step overlap the kernels of the
+        neighbouring steps (what a serving loop does with its input and output staging)."""
+        if getattr(self, "ctx2", None) is not None:
+            return
+        moe, sh, device = self.moe, self.sh, self.device
+        dev = lambda t: None if t is None else t.to(device)
+        self.ctx2 = moe.Context(sh.E, sh.k, sh.H, sh.I, max(T for _, T in self.spec.ops),
+                                max_ops=len(self.spec.ops),
+                                dtype=moe.MOE_DTYPE_FP8_E4M3 if self.fp8 else moe.MOE_DTYPE_BF16, device=device)
+        n_sets = len(self.W)
+        self.layers2 = []
+        for layer, (ops, bound, host) in enumerate(self.layers):
+            W = self.W[layer % n_sets]
+            b2 = []
+            for op, (hx, hi, hw, hy, hs) in zip(ops, host):
+                b2.append(self.ctx2.bind(op.cls, hx.to(device), hi.to(device), hw.to(device), W.w_gate_up, W.w_down,
+                                         x_scale=dev(hs), s_gate_up=W.s_gate_up, s_down=W.s_down))
+            self.layers2.append((ops, b2, host))
+        self.s_h2d, self.s_comp, self.s_d2h = (torch.cuda.Stream(device=device) for _ in range(3))
+
+    def run_e2e(self, steps: int):
+        """`steps` steps with host buffers: every step copies its inputs from pinned host memory,
+        plans, runs and copies its result back to pinned host memory.  Copies and kernels run on
+        three streams over two sets of device buffers; a set is reused only after its results have
+        left the device.  Returns when everything has finished."""
+        self._second_set()
+        sets = [(self.ctx, self.layers), (self.ctx2, self.layers2)]
+        free = {}
+        for step in range(steps):
+            ctx, layers = sets[step % 2]
+            for li, (_, bound, host) in enumerate(layers):
+                key = (step % 2, li)
+                with torch.cuda.stream(self.s_h2d):
+                    if key in free:
+                        self.s_h2d.wait_event(free[key])
+                    for b, (hx, hi, hw, hy, hs) in zip(bound, host):
+                        b.x.copy_(hx, non_blocking=True)
+                        if hs is not None:
+                            b.x_scale.copy_(hs, non_blocking=True)
+                        b.topk_ids.copy_(hi, non_blocking=True)
+                        b.topk_w.copy_(hw, non_blocking=True)
+                    e_in = torch.cuda.Event()
+                    e_in.record(self.s_h2d)
+                with torch.cuda.stream(self.s_comp):
+                    self.s_comp.wait_event(e_in)
+                    if self.spec.layers > 1:
+                        ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
+                    for s_, b in enumerate(bound):
+                        ctx.plan(s_, b)
+                    ctx.run(list(range(len(bound))), fuse_combine=True)
+                    e_run = torch.cuda.Event()
+                    e_run.record(self.s_comp)
+                with torch.cuda.stream(self.s_d2h):
+                    self.s_d2h.wait_event(e_run)
+                    for b, (_, _, _, hy, _) in zip(bound, host):
+                        hy.copy_(b.y, non_blocking=True)
+                    e_out = torch.cuda.Event()
+                    e_out.record(self.s_d2h)
+                free[key] = e_out
+        torch.cuda.synchronize(self.device)
 
 
 def oracle_sample(w: Workload, seconds_target: float = 12.0):
@@ -388,20 +432,17 @@ def run_ours(args):
     value = dist.job_throughput(w.flops * K, secs) / 1e12
     ms_per_step = 1e3 * dist.reduce_scalar(secs, "max") / K
 
-    # ---- end to end with host buffers
-    for _ in range(min(Wm, 3)):
-        w.step_e2e()
+    # ---- end to end with host buffers (host clock around K steps, everything synchronised on both sides)
+    w.run_e2e(min(Wm, 3))
     dist.barrier()
     torch.cuda.synchronize()
-    s2, t2 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    s2.record()
-    for _ in range(K):
-        w.step_e2e()
-    t2.record()
-    torch.cuda.synchronize()
+    t_e2e = time.perf_counter()
+    w.run_e2e(K)
+    t_e2e = time.perf_counter() - t_e2e
     dist.barrier()
     w.ctx.check()
-    e2e_value = dist.job_throughput(w.flops * K, s2.elapsed_time(t2) / 1e3) / 1e12
+    w.ctx2.check()
+    e2e_value = dist.job_throughput(w.flops * K, t_e2e) / 1e12
 
     # ---- roofline of the dominant kernel (the persistent kernel), from live CUDA events
     launches = len(run_ms)
