@@ -126,6 +126,30 @@ def test_small_configs_match_oracle(spec, fuse):
         assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
+@pytest.mark.parametrize("n_ctas", [0, 3], ids=["cta_pairs", "single_ctas"])
+def test_row_counts_at_every_tile_boundary_match_oracle(n_ctas):
+    """Experts whose row counts sit on and around every tile boundary of the run kernels (the 64-row
+    halves of a 128-row MMA over a CTA pair, 128-row m-tiles, 256-row work tiles), full outputs
+    against the oracle, on CTA pairs and on single CTAs."""
+    cnts = [1, 63, 64, 65, 127, 128, 129, 191, 192, 193, 255, 256, 257, 300, 0, 513]
+    E, k, H, I = len(cnts), 1, 512, 256
+    ids = np.concatenate([np.full(c, e) for e, c in enumerate(cnts)]).astype(np.int32)
+    rng = np.random.default_rng(17)
+    ids = ids[rng.permutation(ids.size)].reshape(-1, 1)
+    T = ids.shape[0]
+    spec = synth.Spec("bounds", synth.Shape(E, k, H, I), ((synth.PREFILL, T),), "uniform", None, 1.0, -1.0, 23)
+    W = synth.make_weights(spec)
+    x, _ = synth.make_x(spec, T, 0, 0)
+    op = synth.Op(synth.PREFILL, x, ids, np.ones((T, 1), np.float32))
+    ctx, bound, _, _ = _run_spec(spec, True, ops=[op], W=W, n_ctas=n_ctas)
+    assert ctx.ctas_per_tile == (2 if n_ctas == 0 else 1)
+    counts = check_plan(bound[0], op, E)
+    assert counts.tolist() == cnts
+    check_tiles(ctx, 0, counts)
+    ref = oracle.forward(oracle_weights(spec, W), op.x, None, op.ids, op.w)
+    assert_close(bound[0].y.float().cpu().numpy(), ref["y"])
+
+
 def test_c1_as_stated():
     """C1 with its stated N(0, 0.02) tensors: outputs are ~1e-5, so the absolute term of the
     tolerance is void; the relative-L2 bound is what checks it."""
