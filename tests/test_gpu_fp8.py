@@ -49,6 +49,26 @@ def test_small_fp8_matches_mirrored_oracle(shape):
         assert rel < 8e-2, rel          # information: distance to the un-mirrored reference
 
 
+def test_fp8_row_counts_at_every_tile_boundary():
+    """Expert row counts on and around the 128-row tile boundary of the e4m3 path (and an empty
+    expert), full outputs against the mirrored oracle."""
+    cnts = [1, 7, 8, 9, 127, 128, 129, 255, 256, 257, 0, 300]
+    E, k = len(cnts), 1
+    shape = synth.Shape(E, k, 512, 256, "fp8")
+    ids = np.concatenate([np.full(c, e) for e, c in enumerate(cnts)]).astype(np.int32)
+    ids = ids[np.random.default_rng(3).permutation(ids.size)].reshape(-1, 1)
+    T = ids.shape[0]
+    spec = synth.Spec("fp8b", shape, ((synth.PREFILL, T),), "uniform", None, 1.0, -1.0, 34)
+    W = synth.make_weights(spec)
+    x, xs = synth.make_x(spec, T, 0, 0)
+    op = synth.Op(synth.PREFILL, x, ids, np.ones((T, 1), np.float32), xs)
+    ctx, bound, _, _ = _run(spec, ops=[op], W=W)
+    counts = check_plan(bound[0], op, E)
+    assert counts.tolist() == cnts
+    ref = oracle.forward(oracle_weights(spec, W), op.x, op.x_scale, op.ids, op.w, round_A=oracle.ROUND_E4M3_1X128)
+    assert_close(bound[0].y.float().cpu().numpy(), ref["y"], atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
+
+
 def test_fp8_schedule_independence_bitwise():
     spec = synth.Spec("fp8s", synth.Shape(8, 2, 512, 256, "fp8"), ((synth.PREFILL, 300), (synth.DECODE, 37)),
                       "softmax_topk", None, 1.0, -1.0, 32)
