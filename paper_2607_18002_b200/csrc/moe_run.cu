@@ -97,6 +97,18 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
     sw0 = op->s_down + ((size_t)ti.expert * HB + 2 * ti.n) * IB;
     sw1 = sw0 + IB;
   }
+  if (q * 32 >= ti.rows) {
+    // No row of the tile lies in this warp's TMEM lane quadrant (both warps of a quadrant see
+    // the same q): nothing to read, scale or store.  The warp still takes part in every partial
+    // buffer hand-off, so that the barrier counts and phases stay those of a full tile.
+    for (int kb = 0; kb < ti.kblocks; ++kb) {
+      const int pb = kb & 1;
+      if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->pfull[pb], (eph >> pb) & 1u, 19))) return false;
+      eph ^= 1u << pb;
+      if (lane == 0) mbar_arrive(&sc->pempty[pb]);
+    }
+    return true;
+  }
   float acc[128];                                 // [half][64]
 #pragma unroll
   for (int i = 0; i < 128; ++i) acc[i] = 0.f;
