@@ -372,4 +372,43 @@ __device__ __forceinline__ bool pair_mma_kblock(unsigned d_tmem, unsigned long l
       : "memory");
   return ready != 0;
 }
+// One e4m3 k-block (128 elements = four 32-element MMAs) into a fresh partial buffer, then the two
+// commits (partial full, stage empty), as one group.  Whole warp, warp-uniform operands; one elected
+// lane issues: instructions issued from a divergent single-lane branch cost about 100 clocks each.
+__device__ __forceinline__ void f8_mma_kblock(unsigned d_tmem, unsigned long long adesc, unsigned long long bdesc,
+                                              unsigned idesc, unsigned pfull_bar, unsigned empty_bar) {
+  asm volatile(
+      "{\n\t.reg .pred e, p0, p1;\n\t.reg .b32 r;\n\t.reg .b64 a1, a2, a3, b1, b2, b3;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "setp.ne.b32 p0, 0, 0;\n\t"
+      "setp.eq.b32 p1, 0, 0;\n\t"
+      "add.u64 a1, %1, 2;\n\tadd.u64 a2, %1, 4;\n\tadd.u64 a3, %1, 6;\n\t"
+      "add.u64 b1, %2, 2;\n\tadd.u64 b2, %2, 4;\n\tadd.u64 b3, %2, 6;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], %1, %2, %3, p0;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], a1, b1, %3, p1;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], a2, b2, %3, p1;\n\t"
+      "@e tcgen05.mma.cta_group::1.kind::f8f6f4 [%0], a3, b3, %3, p1;\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%4];\n\t"
+      "@e tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%5];\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(pfull_bar), "r"(empty_bar)
+      : "memory");
+}
+// The loads of one k-block of the single-CTA kernel as ONE group: expect_tx, the two halves of the
+// weight tile and (down tiles) the box of packed intermediate rows.  Whole warp, warp-uniform
+// operands; one elected lane issues.
+__device__ __forceinline__ void single_issue_kblock(unsigned bar, unsigned tx, unsigned sB0, unsigned sB1,
+                                                    const CUtensorMap* tmw, int x, int wy0, int wy1, unsigned sA,
+                                                    const CUtensorMap* tma, int ay, unsigned has_a) {
+  asm volatile(
+      "{\n\t.reg .pred e, pa;\n\t.reg .b32 r;\n\t"
+      "elect.sync r|e, 0xffffffff;\n\t"
+      "setp.ne.and.b32 pa, %11, 0, e;\n\t"
+      "@e mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n\t"
+      "@e cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%2], [%4, {%5, %6}], [%0];\n\t"
+      "@e cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%3], [%4, {%5, %7}], [%0];\n\t"
+      "@pa cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%8], [%9, {%5, %10}], [%0];\n\t}"
+      ::"r"(bar), "r"(tx), "r"(sB0), "r"(sB1), "l"(reinterpret_cast<unsigned long long>(tmw)), "r"(x), "r"(wy0),
+        "r"(wy1), "r"(sA), "l"(reinterpret_cast<unsigned long long>(tma)), "r"(ay), "r"(has_a)
+      : "memory");
+}
 }  // namespace moe

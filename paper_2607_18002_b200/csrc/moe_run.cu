@@ -339,18 +339,11 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         bool fail = false;
         for (int kb = 0; kb < ti.kblocks; ++kb) {
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ph ^ 1u, 5))) { fail = true; break; }
-          if (lane == 0) {
-#ifdef MOE_TIMING_PROBE
-            if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 0] = clock64();
-#endif
-            unsigned char* sA = stages + (size_t)stage * kSB;
-            unsigned char* sB = sA + kBOff;
-            mbar_expect_tx(&sc->full[stage], tx);
-            tma_tile_2d(sB, tmw, kb * kKb, wrow0, &sc->full[stage]);
-            tma_tile_2d(sB + kBHalfBytes, tmw, kb * kKb, wrow1, &sc->full[stage]);
-            if (!g1) tma_tile_2d(sA, tma, kb * kKb, ti.row0, &sc->full[stage]);
+          {
+            const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
+            single_issue_kblock(smem_u32(&sc->full[stage]), tx, sA + kBOff, sA + kBOff + kBHalfBytes, tmw, kb * kKb,
+                                wrow0, wrow1, sA, tma, ti.row0, g1 ? 0u : 1u);
           }
-          __syncwarp();
           if (++stage == kNS) { stage = 0; ph ^= 1u; }
           if (kb == claim_at)              // claim ahead (never blocks here)
             have_nx = claim_once(c, &sc->qt, rh, lane, nx, nx_need_ready) == 1;
@@ -439,18 +432,15 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
               pp[0] = q0; pp[1] = q1; pp[2] = q2; pp[3] = clock64();
             }
 #endif
-            if (lane == 0) {
+            {
               fence_async_proxy_smem();
               const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
               const unsigned long long ad = umma_desc(sA, kRowBytes);
               const unsigned long long bd = umma_desc(sA + kBOff, kRowBytes);
-#pragma unroll
-              for (int k4 = 0; k4 < 4; ++k4)              // 32 e4m3 elements (32 bytes) per step
-                tc_mma_f8(tmem + (unsigned)(pb * 256), ad + 2ull * k4, bd + 2ull * k4, kIdescF8, k4 ? 1u : 0u);
-              tc_commit(&sc->pfull[pb]);
-              tc_commit(&sc->empty[stage]);
+              // four MMAs of 32 e4m3 elements (32 bytes) each, partial full, stage empty
+              f8_mma_kblock(tmem + (unsigned)(pb * 256), ad, bd, kIdescF8, smem_u32(&sc->pfull[pb]),
+                            smem_u32(&sc->empty[stage]));
             }
-            __syncwarp();
           }
           if (fail) break;
           if (++stage == kNS) { stage = 0; ph ^= 1u; }
