@@ -61,7 +61,8 @@ typedef struct {
   int32_t inter;             /* I, multiple of 128                                       */
   int32_t dtype;             /* MOE_DTYPE_*                                              */
   int32_t max_tokens_per_op; /* sizes the per-slot scratch; buffers are fixed up front,  */
-  int32_t max_ops;           /* as the paper's preallocated final buffers (Section 5.2)  */
+  int32_t max_ops;           /* as the paper's preallocated final buffers (Section 5.2); */
+                             /* max_tokens_per_op * k * H must stay below 2^35           */
   int32_t wait_limit_us;     /* device-side wait budget before MOE_ETIMEOUT; 0 = 2 s     */
   int32_t tile_log_entries;  /* capacity of the per-tile log; 0 = logging off            */
   int32_t n_ctas;            /* persistent grid size; 0 = one CTA per SM                 */

@@ -8,12 +8,28 @@
 namespace moe {
 
 // Tokens [t0, t1) by `nthr` cooperating threads (thread index tid); 8 bf16 per 16-byte access.
-// One item = one 16-byte column slice of one token: the token's k rows of D are fetched
-// together (k <= 8: all at once, else eight at a time), so a thread keeps eight 16-byte loads
-// in flight, and the routed rows / router weights of the thread's NEXT item are loaded before
-// the current item's rows are consumed: the two dependent loads of an item (row index, then
-// row) never sit in one latency chain.  The rows are still ADDED in slot order j = 0..k-1.
-__device__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, int H, int tid,
+// k <= 8: a group of L adjacent threads (L = 16, 32, ... as many as the thread count allows)
+// owns one token, loads its k routed rows and router weights once, and walks the token's row in
+// steps of L 16-byte slices.  Slots 0..3 and 4..7 are two buffers: as soon as one has been added
+// in, its loads for the next slice are issued, so loads are in flight all the time and the
+// dependent pair (row index, then row) is paid once per token.  The rows are ADDED in slot
+// order j = 0..k-1.
+__device__ __forceinline__ void combine_add4(float (&acc)[8], const uint4 (&d)[4], const float* wj, int n) {
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    if (i < n) {
+      const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&d[i]);
+#pragma unroll
+      for (int c = 0; c < 4; ++c) {
+        const float2 f = __bfloat1622float2(h[c]);
+        acc[2 * c] = fmaf(wj[i], f.x, acc[2 * c]);
+        acc[2 * c + 1] = fmaf(wj[i], f.y, acc[2 * c + 1]);
+      }
+    }
+  }
+}
+
+__device__ __noinline__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, int H, int tid,
                                       int nthr) {
   const int vec_per_row = H / 8;
   const uint4* D = reinterpret_cast<const uint4*>(op->D);
@@ -21,58 +37,58 @@ __device__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, in
   const int* f2s = op->flat_to_sorted;
   const float* w = op->topk_w;
   const int total = (t1 - t0) * vec_per_row;
-  if (k <= 8) {
-    int pj[8];
-    float wj[8];
-    int t_have = -1;
-    auto load_meta = [&](int t) {             // rows and weights of token t
+  if (k <= 8 && nthr >= 16 && vec_per_row % 16 == 0) {
+    int L = 16;
+    while (2 * L * (t1 - t0) <= nthr && vec_per_row % (2 * L) == 0) L *= 2;
+    const int tpp = nthr / L;                 // tokens per pass
+    const int sub = tid % L, trow = tid / L;
+    if (trow >= tpp) return;
+    const int nslice = vec_per_row / L;
+    for (int t = t0 + trow; t < t1; t += tpp) {
+      // row offsets in 16-byte units (moe_create rejects shapes whose D buffer exceeds 2^32 units)
+      unsigned off[8];
+      float wj[8];
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
-        pj[i] = 0;
+        off[i] = 0u;
         wj[i] = 0.f;
         if (i < k) {
-          pj[i] = f2s[(size_t)t * k + i];
+          off[i] = (unsigned)f2s[(size_t)t * k + i] * (unsigned)vec_per_row;
           wj[i] = w[(size_t)t * k + i];
         }
       }
-      t_have = t;
-    };
-    if (tid < total) load_meta(t0 + tid / vec_per_row);
-    for (int idx = tid; idx < total; idx += nthr) {
-      const int t = t0 + idx / vec_per_row, v = idx % vec_per_row;
-      uint4 d[8];
-      float wc[8];
+      const uint4* src = D + sub;
+      uint4* dst = y + (size_t)t * vec_per_row + sub;
+      const int na = k < 4 ? k : 4, nb = k - na;          // slots in the two buffers
+      uint4 da[4], db[4];
 #pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        wc[i] = wj[i];
-        d[i] = make_uint4(0u, 0u, 0u, 0u);
-        if (i < k) d[i] = D[(size_t)pj[i] * vec_per_row + v];
+      for (int i = 0; i < 4; ++i) {
+        da[i] = make_uint4(0u, 0u, 0u, 0u);
+        db[i] = make_uint4(0u, 0u, 0u, 0u);
+        if (i < na) da[i] = src[off[i]];
+        if (i < nb) db[i] = src[off[4 + i]];
       }
-      const int nidx = idx + nthr;
-      if (nidx < total) {
-        const int nt = t0 + nidx / vec_per_row;
-        if (nt != t_have) load_meta(nt);       // issued while the eight row loads above are in flight
+      for (int sl = 0; sl < nslice; ++sl) {
+        const bool more = sl + 1 < nslice;
+        src += L;
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        combine_add4(acc, da, wj, na);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (i < na && more) da[i] = src[off[i]];
+        combine_add4(acc, db, wj + 4, nb);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+          if (i < nb && more) db[i] = src[off[4 + i]];
+        uint4 o;
+        __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
+        *dst = o;
+        dst += L;
       }
-      float acc[8];
-#pragma unroll
-      for (int i = 0; i < 8; ++i) acc[i] = 0.f;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        if (i < k) {
-          const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&d[i]);
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const float2 f = __bfloat1622float2(h[c]);
-            acc[2 * c] = fmaf(wc[i], f.x, acc[2 * c]);
-            acc[2 * c + 1] = fmaf(wc[i], f.y, acc[2 * c + 1]);
-          }
-        }
-      }
-      uint4 o;
-      __nv_bfloat162* oh = reinterpret_cast<__nv_bfloat162*>(&o);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) oh[i] = __floats2bfloat162_rn(acc[2 * i], acc[2 * i + 1]);
-      y[(size_t)t * vec_per_row + v] = o;
     }
     return;
   }

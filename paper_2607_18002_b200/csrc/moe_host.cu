@@ -43,6 +43,8 @@ int check_config(const moe_config_t* c) {
   if (c->dtype != MOE_DTYPE_BF16 && c->dtype != MOE_DTYPE_FP8_E4M3) return MOE_EINVAL;
   if (c->max_tokens_per_op < 1 || c->max_ops < 1 || c->max_ops > kMaxOps) return MOE_EINVAL;
   if ((long long)c->max_tokens_per_op * c->top_k > (1 << 20) * (long long)kTileM) return MOE_EINVAL;
+  // the combine addresses the rows of the down-GEMM output by 32-bit offsets in 16-byte units
+  if ((long long)c->max_tokens_per_op * c->top_k * (c->hidden / 8) >= (1ll << 32)) return MOE_EINVAL;
   if (c->wait_limit_us < 0 || c->tile_log_entries < 0 || c->n_ctas < 0) return MOE_EINVAL;
   return MOE_OK;
 }
