@@ -356,7 +356,44 @@ def tile_stats(w: Workload):
             out["decode_tile_p99_ratio"] = out["corun"]["decode_tile"]["p99_us"] / iso["decode_tile"]["p99_us"]
             out["decode_tile_p50_ratio"] = out["corun"]["decode_tile"]["p50_us"] / iso["decode_tile"]["p50_us"]
             out["decode_op_ratio"] = out["corun"]["decode_op_us"] / iso["decode_op_us"]
+        out["decode_arrives_mid_prefill"] = _mid_run_arrival(w, bound, dec)
     return out
+
+
+def _mid_run_arrival(w: Workload, bound, dec):
+    """The decode op becomes ready while the prefill op of the same launch is being served: its
+    ready word is the prefill op's notify word, which the kernel sets once a third of the prefill
+    tiles have committed.  Reports the time from that commit to the first decode claim (the
+    preemption delay, bounded by the tile a unit runs plus the one it claimed ahead) next to the
+    prefill tile times."""
+    pre = [s for s in range(len(bound)) if s not in dec]
+    ps, ds = pre[0], dec[0]
+    word = torch.zeros(1, dtype=torch.int32, device=w.device)
+    n_pre = w.ctx.footprint(ps)[1]
+    after = max(1, n_pre // 3)
+    bp, bd = bound[ps], bound[ds]
+    bp.c.notify, bp.c.notify_after, bd.c.ready = word.data_ptr(), after, word.data_ptr()
+    try:
+        w.ctx.plan(ps, bp)
+        w.ctx.plan(ds, bd)
+        w.ctx.run([ps, ds], fuse_combine=True)
+        w.ctx.check()
+        log = w.ctx.tile_log()
+    finally:
+        bp.c.notify, bp.c.notify_after, bd.c.ready = None, 0, None
+        w.ctx.plan(ps, bp)
+        w.ctx.plan(ds, bd)
+    p, d = log[log["slot"] == ps], log[log["slot"] == ds]
+    t_ready = int(np.sort(p["t_commit"])[after - 1])
+    first = int(d["t_claim"].min())
+    gemm = p[p["kind"] < 2]
+    service = (gemm["t_commit"].astype(np.int64) - gemm["t_claim"].astype(np.int64)) / 1e3
+    dsvc = (d["t_commit"].astype(np.int64) - d["t_claim"].astype(np.int64))[d["kind"] < 2] / 1e3
+    return {"ready_after_prefill_tiles": int(after), "prefill_tiles": int(n_pre),
+            "ready_to_first_decode_claim_us": (first - t_ready) / 1e3,
+            "prefill_tile_p50_us": float(np.percentile(service, 50)), "prefill_tile_p99_us": float(np.percentile(service, 99)),
+            "decode_tile_p50_us": float(np.percentile(dsvc, 50)), "decode_tile_p99_us": float(np.percentile(dsvc, 99)),
+            "decode_op_us": float((int(d["t_commit"].max()) - t_ready) / 1e3)}
 
 
 # ------------------------------------------------------------------ arms

@@ -87,6 +87,10 @@ typedef struct {
   const uint32_t* ready;  /* optional: the op may be scheduled once *ready != 0           */
   uint32_t* done;         /* optional: set to 1 when the op's last tile has committed     */
   int32_t after_op;       /* -1, or a slot (of the same moe_run) that must finish first   */
+  int32_t notify_after;   /* with `notify`: 1 .. the op's tile count                      */
+  uint32_t* notify;       /* optional: set to 1 (system scope) once notify_after tiles of */
+                          /* this op have committed -- e.g. the ready word of another op, */
+                          /* which then arrives while this one is being served            */
 } moe_op_t;
 
 /* One record per executed tile (only when tile_log_entries > 0). Times are GPU

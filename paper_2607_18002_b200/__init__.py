@@ -55,7 +55,7 @@ class moe_op_t(C.Structure):
                 ("counts", C.c_void_p), ("offsets", C.c_void_p),
                 ("sorted_to_flat", C.c_void_p), ("flat_to_sorted", C.c_void_p),
                 ("ready", C.c_void_p), ("done", C.c_void_p),
-                ("after_op", C.c_int32)]
+                ("after_op", C.c_int32), ("notify_after", C.c_int32), ("notify", C.c_void_p)]
 
 
 class moe_tile_rec_t(C.Structure):
@@ -255,7 +255,7 @@ class BoundOp:
 
 def bind_op(cls: int, x, topk_ids, topk_w, w_gate_up, w_down, top_k: int, n_experts: int,
             x_scale=None, s_gate_up=None, s_down=None, ready=None, done=None,
-            after_op: int = -1) -> BoundOp:
+            after_op: int = -1, notify=None, notify_after: int = 0) -> BoundOp:
     """Fills a moe_op_t from device tensors and allocates its outputs (y and the plan)."""
     import torch
     T = int(topk_ids.shape[0])
@@ -268,11 +268,12 @@ def bind_op(cls: int, x, topk_ids, topk_w, w_gate_up, w_down, top_k: int, n_expe
     f2s = torch.empty(max(T * top_k, 1), dtype=torch.int32, device=dev)
     keep = dict(x=x, x_scale=x_scale, topk_ids=topk_ids, topk_w=topk_w, w_gate_up=w_gate_up,
                 w_down=w_down, s_gate_up=s_gate_up, s_down=s_down, y=y, counts=counts,
-                offsets=offsets, sorted_to_flat=s2f, flat_to_sorted=f2s, ready=ready, done=done)
+                offsets=offsets, sorted_to_flat=s2f, flat_to_sorted=f2s, ready=ready, done=done,
+                notify=notify)
     c_op = moe_op_t(cls, T, _ptr(x), _ptr(x_scale), _ptr(topk_ids), _ptr(topk_w),
                     _ptr(w_gate_up), _ptr(w_down), _ptr(s_gate_up), _ptr(s_down), _ptr(y),
                     _ptr(counts), _ptr(offsets), _ptr(s2f), _ptr(f2s), _ptr(ready), _ptr(done),
-                    after_op)
+                    after_op, notify_after, _ptr(notify))
     return BoundOp(c_op, keep)
 
 

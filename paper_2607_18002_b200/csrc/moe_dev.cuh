@@ -80,6 +80,8 @@ struct __align__(128) OpDev {
   int* flat_to_sorted;
   const unsigned* ready;
   unsigned* done;
+  unsigned* notify;      // set once notify_after tiles of the op have committed
+  int notify_after;
   // workspace-owned
   __nv_bfloat16* A;      // [Rmax, I]  SwiGLU output, packed order (e4m3 bytes in the fp8 path)
   float* a_scale;        // [Rmax, I/128] fp32 scales of A (fp8 path)

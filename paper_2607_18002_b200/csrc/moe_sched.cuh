@@ -232,6 +232,7 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
   if (ti.kind == kGateUp) atomicAdd(&op->g1_done[ti.m], 1);
   if (ti.kind != kCombine) atomicAdd(&op->run->gemm_done, 1);
   const int done = atomicAdd(&op->run->tiles_done, 1) + 1;
+  if (op->notify != nullptr && done == op->notify_after) st_release_sys(op->notify, 1u);
   if (done == op_total_tiles(op, a->fuse_combine)) {
     __threadfence();
     atomicExch(&op->run->done, 1);

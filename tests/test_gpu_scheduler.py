@@ -65,6 +65,54 @@ def test_decode_first_inside_the_budget_and_work_conserving():
     assert len(np.unique(log["cta"])) == units
 
 
+def test_decode_op_that_arrives_mid_prefill_is_served_within_the_preemption_bound():
+    """Section 4.3: a phase switch happens only at a tile boundary, so a decode operation that
+    becomes ready while prefill tiles run is first served after at most the tile a unit executes
+    plus the one it had claimed ahead.  The decode op's ready word is the prefill op's notify
+    word, set by the kernel itself when a third of the prefill tiles have committed."""
+    W = weights_to(synth.make_weights(SPEC))
+    ops = synth.make_ops(SPEC)
+    ctx = make_ctx(SPEC, max_tokens=4096, max_ops=2, tile_log_entries=1 << 15)
+    # reference run: both ops ready at launch
+    plain = bind_ops(ctx, ops, W)
+    for s, b in enumerate(plain):
+        ctx.plan(s, b)
+    ctx.run([0, 1], fuse_combine=True)
+    ctx.check()
+    y_ref = [b.y.clone() for b in plain]
+    n_pre = ctx.footprint(0)[1]
+    # the same ops, the decode op gated by the prefill op's progress
+    word = torch.zeros(1, dtype=torch.int32, device="cuda:0")
+    from gpu_util import upload
+    d0, d1 = upload(ops[0], None, "cuda:0"), upload(ops[1], None, "cuda:0")
+    after = n_pre // 3
+    pre = ctx.bind(ops[0].cls, d0["x"], d0["ids"], d0["w"], W.w_gate_up, W.w_down, notify=word, notify_after=after)
+    dec = ctx.bind(ops[1].cls, d1["x"], d1["ids"], d1["w"], W.w_gate_up, W.w_down, ready=word)
+    ctx.set_budget(32)
+    ctx.plan(0, pre)
+    ctx.plan(1, dec)
+    ctx.run([0, 1], fuse_combine=True)
+    ctx.check()
+    log = ctx.tile_log()
+    assert int(word.item()) == 1
+    # results do not depend on when the decode op arrived
+    assert torch.equal(pre.y, y_ref[0]) and torch.equal(dec.y, y_ref[1])
+    p, d = log[log["cls"] == 1], log[log["cls"] == 0]
+    assert len(d) == ctx.footprint(1)[1]
+    t_ready = np.sort(p["t_commit"])[after - 1]           # the commit that set the word
+    # no decode tile was handed out before the word was set ...
+    first = d["t_claim"].min()
+    assert first >= t_ready - 2000                        # the log stamp precedes the store by a few hundred ns
+    # ... and the first one within two prefill tile times of it
+    service = (p["t_commit"].astype(np.int64) - p["t_claim"].astype(np.int64))[p["kind"] < 2]
+    assert first - t_ready <= 2 * np.percentile(service, 99)
+    # from then on the units inside the budget serve decode tiles
+    q_units = 32 // ctx.ctas_per_tile
+    t_dec_end = d["t_claim"].max()
+    inside = log[(log["cta"] < 32) & (log["t_claim"] > first) & (log["t_claim"] < t_dec_end)]
+    assert (inside["cls"] == 1).sum() <= 2 * q_units
+
+
 def test_single_class_uses_all_ctas():
     ctx, log = _run(budget=16, n_ops=1)          # only the prefill op: decode budget must not idle CTAs
     assert len(np.unique(log["cta"])) == ctx.sm_count // ctx.ctas_per_tile
