@@ -91,6 +91,9 @@ typedef struct {
   uint32_t* notify;       /* optional: set to 1 (system scope) once notify_after tiles of */
                           /* this op have committed -- e.g. the ready word of another op, */
                           /* which then arrives while this one is being served            */
+  int32_t decode_sms;     /* the SM budget field of the op template (Section 4.2): > 0    */
+                          /* makes the decode budget take this value when the op's first  */
+                          /* tile is claimed, 0 leaves the budget word alone              */
 } moe_op_t;
 
 /* One record per executed tile (only when tile_log_entries > 0). Times are GPU

@@ -55,7 +55,8 @@ class moe_op_t(C.Structure):
                 ("counts", C.c_void_p), ("offsets", C.c_void_p),
                 ("sorted_to_flat", C.c_void_p), ("flat_to_sorted", C.c_void_p),
                 ("ready", C.c_void_p), ("done", C.c_void_p),
-                ("after_op", C.c_int32), ("notify_after", C.c_int32), ("notify", C.c_void_p)]
+                ("after_op", C.c_int32), ("notify_after", C.c_int32), ("notify", C.c_void_p),
+                ("decode_sms", C.c_int32)]
 
 
 class moe_tile_rec_t(C.Structure):
@@ -255,7 +256,7 @@ class BoundOp:
 
 def bind_op(cls: int, x, topk_ids, topk_w, w_gate_up, w_down, top_k: int, n_experts: int,
             x_scale=None, s_gate_up=None, s_down=None, ready=None, done=None,
-            after_op: int = -1, notify=None, notify_after: int = 0) -> BoundOp:
+            after_op: int = -1, notify=None, notify_after: int = 0, decode_sms: int = 0) -> BoundOp:
     """Fills a moe_op_t from device tensors and allocates its outputs (y and the plan)."""
     import torch
     T = int(topk_ids.shape[0])
@@ -273,7 +274,7 @@ def bind_op(cls: int, x, topk_ids, topk_w, w_gate_up, w_down, top_k: int, n_expe
     c_op = moe_op_t(cls, T, _ptr(x), _ptr(x_scale), _ptr(topk_ids), _ptr(topk_w),
                     _ptr(w_gate_up), _ptr(w_down), _ptr(s_gate_up), _ptr(s_down), _ptr(y),
                     _ptr(counts), _ptr(offsets), _ptr(s2f), _ptr(f2s), _ptr(ready), _ptr(done),
-                    after_op, notify_after, _ptr(notify))
+                    after_op, notify_after, _ptr(notify), decode_sms)
     return BoundOp(c_op, keep)
 
 

@@ -82,6 +82,7 @@ struct __align__(128) OpDev {
   unsigned* done;
   unsigned* notify;      // set once notify_after tiles of the op have committed
   int notify_after;
+  int op_budget;         // > 0: written to the budget word when the op's first tile is claimed
   // workspace-owned
   __nv_bfloat16* A;      // [Rmax, I]  SwiGLU output, packed order (e4m3 bytes in the fp8 path)
   float* a_scale;        // [Rmax, I/128] fp32 scales of A (fp8 path)

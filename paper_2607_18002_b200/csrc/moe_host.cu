@@ -221,6 +221,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   if (op->n_tokens > c.max_tokens_per_op) return MOE_ENOSPC;
   if (op->after_op < -1 || op->after_op >= c.max_ops || op->after_op == slot) return MOE_EINVAL;
   if (op->notify && op->notify_after < 1) return MOE_EINVAL;
+  if (op->decode_sms < 0) return MOE_EINVAL;
   if (!op->counts || !op->offsets) return MOE_EINVAL;
   if (!op->w_gate_up || !op->w_down || !aligned16(op->w_gate_up) || !aligned16(op->w_down)) return MOE_EINVAL;
   if (c.dtype == MOE_DTYPE_FP8_E4M3 && (!op->s_gate_up || !op->s_down || (op->n_tokens > 0 && !op->x_scale)))
@@ -244,6 +245,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   h.sorted_to_flat = op->sorted_to_flat; h.flat_to_sorted = op->flat_to_sorted;
   h.ready = op->ready; h.done = op->done;
   h.notify = op->notify; h.notify_after = op->notify_after;
+  h.op_budget = op->decode_sms;
   h.A = reinterpret_cast<__nv_bfloat16*>(sb + L.A_off);
   h.a_scale = reinterpret_cast<float*>(sb + L.A_off + align_up((size_t)L.max_rows * c.inter, 16));
   h.D = reinterpret_cast<__nv_bfloat16*>(sb + L.D_off);

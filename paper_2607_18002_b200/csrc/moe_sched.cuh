@@ -139,6 +139,8 @@ __device__ inline int try_claim(const RunArgs* a, QueueTables* sc, RunHead* rh, 
     need_ready = !sc->cls_free[cls][i];
   }
   const unsigned local = t - sc->cum[cls][i];
+  // the op is instantiated by the claim of its first tile: its budget field takes effect now
+  if (local == 0 && lane == 0 && op->op_budget > 0) atomicExch(&a->g->budget, op->op_budget);
   const unsigned d = t - h;
   const bool hit = !need_ready && d < 32u;
   int4 got;

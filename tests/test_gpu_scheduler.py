@@ -113,6 +113,49 @@ def test_decode_op_that_arrives_mid_prefill_is_served_within_the_preemption_boun
     assert (inside["cls"] == 1).sum() <= 2 * q_units
 
 
+def test_one_launch_over_three_layers_with_the_budget_carried_by_the_ops():
+    """A kernel that lives across layers (Section 4.2): six operations in one launch, chained by
+    after_op (prefill l after prefill l-1, decode l after prefill l-1), every decode op carrying its
+    own SM budget.  Results equal the per-layer launches bit for bit."""
+    spec = synth.Spec("layers", SPEC.shape, ((synth.PREFILL, 1024), (synth.DECODE, 64)), "zipf", 1.0, 1.0, -1.0, 43,
+                      layers=3)
+    W = weights_to(synth.make_weights(spec))
+    budgets = (16, 32, 64)
+    small = make_ctx(spec, max_tokens=1024, max_ops=2)
+    y_ref = []
+    for l in range(3):
+        b = bind_ops(small, synth.make_ops(spec, l), W)
+        small.set_budget(budgets[l])
+        for s, x in enumerate(b):
+            small.plan(s, x)
+        small.run([0, 1], fuse_combine=True)
+        small.check()
+        y_ref.append([x.y.clone() for x in b])
+    ctx = make_ctx(spec, max_tokens=1024, max_ops=6, tile_log_entries=1 << 15)
+    from gpu_util import upload
+    bound = []
+    for l in range(3):
+        for j, op in enumerate(synth.make_ops(spec, l)):
+            d = upload(op, None, "cuda:0")
+            bound.append(ctx.bind(op.cls, d["x"], d["ids"], d["w"], W.w_gate_up, W.w_down,
+                                  after_op=(2 * (l - 1) if l > 0 else -1),
+                                  decode_sms=(budgets[l] if op.cls == synth.DECODE else 0)))
+    ctx.set_budget(1)
+    for s, b in enumerate(bound):
+        ctx.plan(s, b)
+    ctx.run(list(range(6)), fuse_combine=True)
+    ctx.check()
+    for l in range(3):
+        assert torch.equal(bound[2 * l].y, y_ref[l][0]) and torch.equal(bound[2 * l + 1].y, y_ref[l][1])
+    assert ctx.get_budget() == budgets[2]                 # the last decode op's field was the last write
+    log = ctx.tile_log()
+    for l in (1, 2):
+        done_prev = log["t_commit"][log["slot"] == 2 * (l - 1)].max()
+        assert log["t_claim"][log["slot"] == 2 * l].min() >= 0      # claimed ahead is allowed ...
+        assert log["t_commit"][log["slot"] == 2 * l].min() >= done_prev     # ... but nothing of it ran before
+        assert log["t_commit"][log["slot"] == 2 * l + 1].min() >= done_prev
+
+
 def test_single_class_uses_all_ctas():
     ctx, log = _run(budget=16, n_ops=1)          # only the prefill op: decode budget must not idle CTAs
     assert len(np.unique(log["cta"])) == ctx.sm_count // ctx.ctas_per_tile
