@@ -396,6 +396,57 @@ def _mid_run_arrival(w: Workload, bound, dec):
             "decode_op_us": float((int(d["t_commit"].max()) - t_ready) / 1e3)}
 
 
+def persistent_layers(w: Workload, steps: int, warmup: int):
+    """The multi-layer workload as ONE persistent launch per step: all ops of all layers in one
+    moe_run, prefill l after prefill l-1 and decode l after prefill l-1 (after_op), every decode op
+    carrying the SM budget of its layer (moe_op_t.decode_sms) -- no launch, no host call and no
+    separate budget write between layers.  Same inputs, same plan calls as the per-layer step."""
+    moe, sh = w.moe, w.sh
+    n_layers = len(w.layers)
+    ctx = moe.Context(sh.E, sh.k, sh.H, sh.I, max(T for _, T in w.spec.ops), max_ops=2 * n_layers,
+                      dtype=moe.MOE_DTYPE_FP8_E4M3 if w.fp8 else moe.MOE_DTYPE_BF16, device=w.device)
+    bound = []
+    for l, (ops, b_old, _) in enumerate(w.layers):
+        W = w.W[l % len(w.W)]
+        prev_prefill = next((2 * (l - 1) + j for j, o in enumerate(w.layers[l - 1][0]) if o.cls == synth.PREFILL), -1) if l else -1
+        for op, b in zip(ops, b_old):
+            bound.append(ctx.bind(op.cls, b.x, b.topk_ids, b.topk_w, W.w_gate_up, W.w_down, x_scale=b.x_scale,
+                                  s_gate_up=W.s_gate_up, s_down=W.s_down, after_op=prev_prefill,
+                                  decode_sms=synth.C4_BUDGETS[l % len(synth.C4_BUDGETS)] if op.cls == synth.DECODE else 0))
+    slots = list(range(len(bound)))
+
+    def step():
+        for s_, b in enumerate(bound):
+            ctx.plan(s_, b)
+        ctx.run(slots, fuse_combine=True)
+
+    for _ in range(warmup):
+        step()
+    ctx.check()
+    torch.cuda.synchronize()
+    # The two forms alternate step by step, so that both see the same clocks (the power limit moves
+    # them over a run of this length).
+    t_one, t_per = [], []
+    for _ in range(steps):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record()
+        step()
+        ev[1].record()
+        w.step()
+        ev[2].record()
+        torch.cuda.synchronize()
+        t_one.append(ev[0].elapsed_time(ev[1]))
+        t_per.append(ev[1].elapsed_time(ev[2]))
+    ctx.check()
+    w.ctx.check()
+    ms = float(np.mean(t_one))
+    same = all(torch.equal(b.y, bo.y) for b, (_, b_old, _) in zip([bound[i:i + 2] for i in range(0, len(bound), 2)], w.layers)
+               for b, bo in zip(b, b_old)) if all(len(x[1]) == 2 for x in w.layers) else None
+    return {"ms_per_step": ms, "value": w.flops / (ms / 1e3) / 1e12, "unit": UNIT, "ops_in_launch": len(bound),
+            "launches_per_step": len(bound) * KERNELS_PER_PLAN + 1, "outputs_equal_per_layer_launches": same,
+            "per_layer_launches_ms_per_step_alternating": float(np.mean(t_per))}
+
+
 # ------------------------------------------------------------------ arms
 
 def run_reference(args):
@@ -513,6 +564,7 @@ def run_ours(args):
                  "hbm_frac": hbm_frac})
 
     tiles = tile_stats(w) if args.tile_log else None
+    one_launch = persistent_layers(w, K, Wm) if (args.one_launch and len(w.layers) > 1 and world == 1) else None
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -534,7 +586,8 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": w.h2d,
                     "d2h_bytes_per_step": w.d2h},
             "gpu_launches": w.launches_per_step * K,
-            "roofline": roof, "cpu_baseline": cpu, **({"tiles": tiles} if tiles else {})}))
+            "roofline": roof, "cpu_baseline": cpu, **({"tiles": tiles} if tiles else {}),
+            **({"one_launch_for_all_layers": one_launch} if one_launch else {})}))
     dist.shutdown()
 
 
@@ -547,6 +600,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tile-log", action="store_true", help="add per-tile timing statistics of one extra untimed step")
+    ap.add_argument("--one-launch", action="store_true",
+                    help="multi-layer workloads: also time all layers as one persistent launch per step")
     args = ap.parse_args()
     ds, dw = DEFAULT_STEPS[args.workload]
     if args.impl == "reference":
