@@ -126,6 +126,21 @@ def test_small_configs_match_oracle(spec, fuse):
         assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
+@pytest.mark.parametrize("fuse", [False, True])
+@pytest.mark.parametrize("k", [1, 3, 6, 12])
+def test_other_top_k_values_match_oracle(k, fuse):
+    """top-k values besides the configs' 2 and 8: the combine splits the k slots into buffers of four
+    (k = 3, 6 leave one partly filled) and takes another path above eight slots."""
+    spec = synth.Spec(f"k{k}", synth.Shape(16, k, 512, 256), ((synth.PREFILL, 200), (synth.DECODE, 9)), "uniform", None,
+                      1.0, -1.0, 29)
+    ctx, bound, ops, W = _run_spec(spec, fuse)
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        ref = oracle.forward(OW, op.x, None, op.ids, op.w)
+        check_plan(b, op, spec.shape.E)
+        assert_close(b.y.float().cpu().numpy(), ref["y"])
+
+
 @pytest.mark.parametrize("n_ctas", [0, 3], ids=["cta_pairs", "single_ctas"])
 def test_row_counts_at_every_tile_boundary_match_oracle(n_ctas):
     """Experts whose row counts sit on and around every tile boundary of the run kernels (the 64-row
