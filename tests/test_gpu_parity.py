@@ -141,6 +141,30 @@ def test_other_top_k_values_match_oracle(k, fuse):
         assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
+def test_shared_expert_as_one_more_slot():
+    """A shared (always-on) expert, Section 2.1: it is expert E-1 here, and every token carries it as
+    one more top-k slot with weight 1 next to its routed experts.  The output is the routed output
+    plus the shared expert's, which the oracle also gives when the two parts run as separate ops."""
+    E, k, H, I, T = 9, 3, 512, 256, 150
+    spec = synth.Spec("shared", synth.Shape(E, k, H, I), ((synth.PREFILL, T),), "uniform", None, 1.0, -1.0, 31)
+    W = synth.make_weights(spec)
+    x, _ = synth.make_x(spec, T, 0, 0)
+    rng = np.random.default_rng(5)
+    routed = np.stack([rng.permutation(E - 1)[:k - 1] for _ in range(T)]).astype(np.int32)
+    wr = rng.random((T, k - 1)).astype(np.float32)
+    wr /= wr.sum(1, keepdims=True)
+    ids = np.concatenate([routed, np.full((T, 1), E - 1, np.int32)], axis=1)
+    w = np.concatenate([wr, np.ones((T, 1), np.float32)], axis=1)
+    op = synth.Op(synth.PREFILL, x, ids, w)
+    ctx, bound, _, _ = _run_spec(spec, True, ops=[op], W=W)
+    OW = oracle_weights(spec, W)
+    ref = oracle.forward(OW, x, None, ids, w)["y"]
+    parts = (oracle.forward(OW, x, None, routed, wr)["y"] +
+             oracle.forward(OW, x, None, ids[:, -1:], w[:, -1:])["y"])
+    np.testing.assert_allclose(ref, parts, rtol=1e-6, atol=1e-6)
+    assert_close(bound[0].y.float().cpu().numpy(), ref)
+
+
 @pytest.mark.parametrize("n_ctas", [0, 3], ids=["cta_pairs", "single_ctas"])
 def test_row_counts_at_every_tile_boundary_match_oracle(n_ctas):
     """Experts whose row counts sit on and around every tile boundary of the run kernels (the 64-row
