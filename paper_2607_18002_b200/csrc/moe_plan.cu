@@ -84,6 +84,7 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   __shared__ int warp_sums[33];
   __shared__ int s_cnt[kMaxExperts], s_grp[kMaxExperts], s_moff[kMaxExperts], s_off[kMaxExperts];
   __shared__ int s_part[1024];
+  __shared__ int s_w0[kMaxExperts];
   __shared__ int g_cnt[kMaxExperts], g_base1[kMaxExperts], g_base2[kMaxExperts];
   __shared__ int s_ntiles;
   const int e = threadIdx.x;
@@ -100,7 +101,7 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   const int c0 = min(n_chunks, part * cpp), c1 = min(n_chunks, c0 + cpp);
   int psum = 0;
   if (part < parts) {
-#pragma unroll 8
+#pragma unroll 32
     for (int c = c0; c < c1; ++c) psum += hist[(size_t)c * E + pe];
     s_part[part * E + pe] = psum;
   }
@@ -121,7 +122,7 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   if (part < parts) {
     int run = s_off[pe];
     for (int p = 0; p < part; ++p) run += s_part[p * E + pe];
-#pragma unroll 8
+#pragma unroll 32
     for (int c = c0; c < c1; ++c) {
       const int v = hist[(size_t)c * E + pe];
       base[(size_t)c * E + pe] = run;
@@ -152,13 +153,15 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   // gate/up tiles of its group and of one more group, so by the time it is claimed the tiles
   // it depends on were claimed long before.
   const int we = (e < E) ? (cnt + work_rows - 1) / work_rows : 0;
+  s_part[e] = we;                 // the column sums are consumed: the array now holds work tiles per expert
   int n_work;
   const int w0 = block_excl_scan(we, &n_work, warp_sums);
+  if (e < E) s_w0[e] = w0;
   __syncthreads();
   if (threadIdx.x == 0) {
     int ng = 0, acc = 0;
     for (int x = 0; x < E; ++x) {
-      const int m = (s_cnt[x] + work_rows - 1) / work_rows;
+      const int m = s_part[x];
       s_grp[x] = ng;
       s_moff[x] = acc;
       acc += m;
@@ -178,14 +181,21 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   }
   __syncthreads();
 
-  if (e < E && we > 0) {           // inside an expert: n-major over its work tiles
-    const int gi = s_grp[e];
-    const int b1 = g_base1[gi] + s_moff[e] * NT1, b2 = g_base2[gi] + s_moff[e] * NT2;
-    for (int j = 0; j < we; ++j) {
-      const int row0 = off + j * work_rows, rows = min(work_rows, cnt - j * work_rows);
-      const int m = w0 + j;
-      for (int n = 0; n < NT1; ++n) op->tile_list[b1 + n * we + j] = make_entry(kGateUp, n, m, row0, rows, e);
-      for (int n = 0; n < NT2; ++n) op->tile_list[b2 + n * we + j] = make_entry(kDown, n, m, row0, rows, e);
+  // Inside an expert: n-major over its work tiles, so an expert's entries of one GEMM are one
+  // contiguous run of the list.  One warp per expert writes them (a popular expert has hundreds).
+  for (int x = threadIdx.x >> 5; x < E; x += 32) {
+    const int wx = s_part[x];
+    if (wx == 0) continue;
+    const int lane = threadIdx.x & 31;
+    const int gi = s_grp[x], cx = s_cnt[x], ox = s_off[x], mx = s_w0[x];
+    const int b1 = g_base1[gi] + s_moff[x] * NT1, b2 = g_base2[gi] + s_moff[x] * NT2;
+    for (int i = lane; i < wx * NT1; i += 32) {
+      const int n = i / wx, j = i - n * wx;
+      op->tile_list[b1 + i] = make_entry(kGateUp, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
+    }
+    for (int i = lane; i < wx * NT2; i += 32) {
+      const int n = i / wx, j = i - n * wx;
+      op->tile_list[b2 + i] = make_entry(kDown, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
     }
   }
   const int n_gemm = s_ntiles;
