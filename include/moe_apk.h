@@ -186,8 +186,9 @@ int moe_read_tile_log(moe_ctx_t* ctx, moe_tile_rec_t* host_out, int max_records,
  *     MOE_PLAN_STATIC_MAX_EXPERTS, else MOE_ENOSPC (nothing is launched);
  *   - all pointers are device pointers owned by the caller, sizes as in moe_op_t;
  *   - expert ids outside [0, n_experts) are skipped silently (moe_plan reports them);
- *   - the first call on each device looks up the scratch array's device address; make
- *     that first call outside any stream capture;
+ *   - every call looks up the scratch array's device address (nothing is cached, so a device
+ *     reset between calls is harmless); the first look-up on a device may load the library's
+ *     device code: make that first call outside any stream capture;
  *   - every call uses the same array, which keeps the previous call's contents (nothing
  *     in it needs clearing between calls); calls whose kernels could overlap on the GPU
  *     -- other streams, other host threads -- race on it and must be serialised. */

@@ -11,16 +11,14 @@
 // scratch is ours.
 //
 // The array's name is a host-side handle in host code, not a device address, so the address
-// is looked up once per device with cudaGetSymbolAddress and that pointer is what the
-// kernels receive.  The look-up happens in the first call on a device; make that first call
-// outside any stream capture.
+// is looked up with cudaGetSymbolAddress and that pointer is what the kernels receive.  The
+// first look-up on a device may load the library's device code; make that first call outside
+// any stream capture.
 //
 // All calls share the one array and it keeps the last call's contents.  Nothing in it has
 // to start at zero (every entry a call reads was written by the same call), but two calls
 // whose kernels overlap on the GPU (different streams, or different host threads) would
 // race on it: serialise them.
-#include <mutex>
-
 #include "moe_dev.cuh"
 
 namespace moe {
@@ -124,21 +122,14 @@ static_scatter_kernel(const int* __restrict__ ids, const int* __restrict__ hist,
   }
 }
 
-// device address of the scratch array on the current device (looked up once per device)
+// Device address of the scratch array on the current device.  Looked up on every call: a cached
+// pointer would dangle once the caller resets the device (the array then moves with the reloaded
+// module), and after the first call the look-up is a table read.
 static int scratch_on_current_device(int** out) {
-  static std::mutex mu;
-  static int* ptr[64] = {nullptr};
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess) return MOE_ECUDA;
-  if (dev < 0 || dev >= 64) return MOE_EINVAL;
-  std::lock_guard<std::mutex> lock(mu);
-  if (ptr[dev] == nullptr) {
-    void* p = nullptr;
-    const cudaError_t e = cudaGetSymbolAddress(&p, g_plan_scratch);
-    if (e != cudaSuccess || p == nullptr) return MOE_ECUDA;
-    ptr[dev] = static_cast<int*>(p);
-  }
-  *out = ptr[dev];
+  void* p = nullptr;
+  const cudaError_t e = cudaGetSymbolAddress(&p, g_plan_scratch);
+  if (e != cudaSuccess || p == nullptr) return MOE_ECUDA;
+  *out = static_cast<int*>(p);
   return MOE_OK;
 }
 
