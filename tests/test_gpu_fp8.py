@@ -49,6 +49,31 @@ def test_small_fp8_matches_mirrored_oracle(shape):
         assert rel < 8e-2, rel          # information: distance to the un-mirrored reference
 
 
+def _random_fp8_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        E = int(rng.integers(1, 33))
+        k = int(rng.integers(1, min(E, 8) + 1))
+        out.append((E, k, int(rng.choice([256, 512, 768])), int(rng.choice([128, 256, 384])), int(rng.integers(1, 500)),
+                    int(rng.integers(0, 50)), str(rng.choice(["uniform", "zipf"])), int(rng.integers(0, 64)), 200 + i))
+    return out
+
+
+@pytest.mark.parametrize("case", _random_fp8_cases(8, 77), ids=lambda c: "E%d_k%d_H%d_I%d_T%d+%d_%s" % c[:7])
+def test_seeded_random_fp8_shapes_match_mirrored_oracle(case):
+    E, k, H, I, T1, T0, routing, budget, seed = case
+    opsdef = ((synth.PREFILL, T1),) + (((synth.DECODE, T0),) if T0 > 0 else ())
+    spec = synth.Spec("rand8", synth.Shape(E, k, H, I, "fp8"), opsdef, routing, 1.0 if routing == "zipf" else None, 1.0, -1.0,
+                      seed)
+    ctx, bound, ops, W = _run(spec, budget=budget)
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        check_plan(b, op, E)
+        ref = oracle.forward(OW, op.x, op.x_scale, op.ids, op.w, round_A=oracle.ROUND_E4M3_1X128)
+        assert_close(b.y.float().cpu().numpy(), ref["y"], atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
+
+
 def test_fp8_row_counts_at_every_tile_boundary():
     """Expert row counts on and around the 128-row tile boundary of the e4m3 path (and an empty
     expert), full outputs against the mirrored oracle."""

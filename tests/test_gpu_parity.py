@@ -141,6 +141,37 @@ def test_other_top_k_values_match_oracle(k, fuse):
         assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
+def _random_cases(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        E = int(rng.integers(1, 41))
+        k = int(rng.integers(1, min(E, 10) + 1))
+        H = int(rng.choice([256, 512, 768, 1024]))
+        I = int(rng.choice([128, 256, 384, 512]))
+        T1, T0 = int(rng.integers(1, 700)), int(rng.integers(0, 60))
+        routing = str(rng.choice(["uniform", "zipf"]))
+        out.append((E, k, H, I, T1, T0, routing, int(rng.choice([0, 0, 3, 8])), int(rng.integers(0, 64)), bool(rng.integers(0, 2)),
+                    100 + i))
+    return out
+
+
+@pytest.mark.parametrize("case", _random_cases(12, 2024), ids=lambda c: "E%d_k%d_H%d_I%d_T%d+%d_%s_g%d" % c[:8])
+def test_seeded_random_shapes_match_oracle(case):
+    """Shapes, token counts, routing, grid size, budget and combine mode drawn from a seeded generator:
+    plan bit-exact, outputs within the bf16 tolerance, for both ops of a co-scheduled batch."""
+    E, k, H, I, T1, T0, routing, n_ctas, budget, fuse, seed = case
+    opsdef = ((synth.PREFILL, T1),) + (((synth.DECODE, T0),) if T0 > 0 else ())
+    spec = synth.Spec("rand", synth.Shape(E, k, H, I), opsdef, routing, 1.0 if routing == "zipf" else None, 1.0, -1.0, seed)
+    ctx, bound, ops, W = _run_spec(spec, fuse, budget=budget, n_ctas=n_ctas)
+    OW = oracle_weights(spec, W)
+    for s_, (b, op) in enumerate(zip(bound, ops)):
+        counts = check_plan(b, op, E)
+        check_tiles(ctx, s_, counts)
+        ref = oracle.forward(OW, op.x, None, op.ids, op.w)
+        assert_close(b.y.float().cpu().numpy(), ref["y"])
+
+
 def test_shared_expert_as_one_more_slot():
     """A shared (always-on) expert, Section 2.1: it is expert E-1 here, and every token carries it as
     one more top-k slot with weight 1 next to its routed experts.  The output is the routed output
