@@ -33,7 +33,7 @@ METRIC = "moe_expert_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 KERNELS_PER_PLAN = 3          # histogram, scan + tile list, scatter
-DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c2s": (20, 3), "c3s": (10, 3), "c5s": (10, 3)}
+DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c2s": (20, 3), "c3s": (10, 3), "c4s": (5, 3), "c5s": (10, 3)}
 
 
 
@@ -46,6 +46,8 @@ NCU_DRAM_BYTES = {
     ("c3", "moe_apk_pair_kernel"): (2.029e9 + 0.160e9) * 256 / 64,
     ("c2s", "moe_apk_pair_kernel"): 1.815e9 + 0.007e9,
     ("c2", "moe_apk_pair_kernel"): (1.815e9 + 0.007e9) * 251 / 63,
+    ("c4s", "moe_apk_pair_kernel"): 4.036e9 + 0.350e9,
+    ("c4", "moe_apk_pair_kernel"): (4.036e9 + 0.350e9) * 256 / 64,
     ("c5s", "moe_apk_kernel"): 2.524e9 + 0.087e9,
     ("c5", "moe_apk_kernel"): (2.524e9 + 0.087e9) * 256 / 32,
 }
@@ -596,7 +598,7 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "c2s", "c3s", "c5s"])
+    ap.add_argument("--workload", default="c3", choices=["c2", "c3", "c4", "c5", "c2s", "c3s", "c4s", "c5s"])
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tile-log", action="store_true", help="add per-tile timing statistics of one extra untimed step")

@@ -96,6 +96,8 @@ SPECS["c2s"] = scaled_ = dataclasses.replace(SPECS["c2"], name="c2s", shape=Shap
                                              ops=((DECODE, 32),))
 SPECS["c3s"] = dataclasses.replace(SPECS["c3"], name="c3s", shape=Shape(64, 8, 3072, 1536),
                                    ops=((PREFILL, 2048),))
+SPECS["c4s"] = dataclasses.replace(SPECS["c4"], name="c4s", shape=Shape(64, 8, 3072, 1536),
+                                   ops=((PREFILL, 4096), (DECODE, 64)), layers=2)
 SPECS["c5s"] = dataclasses.replace(SPECS["c5"], name="c5s", shape=Shape(32, 8, 6144, 2048, "fp8"),
                                    ops=((PREFILL, 512), (DECODE, 64)))
 del scaled_
