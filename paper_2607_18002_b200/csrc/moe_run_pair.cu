@@ -15,9 +15,10 @@
 // Roles per CTA (16 warps): leader only -- warp 0 scheduler (claims, waits for dependencies,
 // publishes tile descriptors to both CTAs), warp 1 MMA issuer, warp 2 committer; both CTAs --
 // warp 3 producer (TMA loads of its own half, read from the descriptor ring), warps 4-7 gather,
-// warps 8-15 epilogue; second CTA only -- warp 1 relays the completion of its gather to the leader.  Tile descriptors reach the second CTA through distributed shared
-// memory; its barrier arrivals that the leader waits for are remote mbarrier arrivals.  Every
-// wait is bounded, as in the single-CTA kernel.
+// warps 8-15 epilogue; second CTA only -- warp 1 relays the completion of its gather to the
+// leader.  Tile descriptors reach the second CTA through distributed shared memory; its barrier
+// arrivals that the leader waits for are remote mbarrier arrivals.  Every wait is bounded, as in
+// the single-CTA kernel.
 #include "moe_combine.cuh"
 #include "moe_ptx.cuh"
 #include "moe_sched.cuh"
