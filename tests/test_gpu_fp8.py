@@ -74,6 +74,27 @@ def test_seeded_random_fp8_shapes_match_mirrored_oracle(case):
         assert_close(b.y.float().cpu().numpy(), ref["y"], atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
 
 
+@pytest.mark.parametrize("case", [(1024, 32, 256, 128, 40, 3, 0), (256, 8, 512, 256, 5000, 300, 0), (5, 2, 256, 128, 3000, 0, 10)],
+                         ids=["E1024_k32", "E256_5000_tokens", "ten_ctas"])
+def test_fp8_limits_of_the_configuration(case):
+    E, k, H, I, T1, T0, n_ctas = case
+    opsdef = ((synth.PREFILL, T1),) + (((synth.DECODE, T0),) if T0 else ())
+    spec = synth.Spec("lim8", synth.Shape(E, k, H, I, "fp8"), opsdef, "zipf", 1.1, 1.0, -1.0, 7)
+    W = synth.make_weights(spec)
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec, max_tokens=max(o.T for o in ops), max_ops=len(ops), n_ctas=n_ctas)
+    bound = bind_ops(ctx, ops, weights_to(W))
+    for s_, b in enumerate(bound):
+        ctx.plan(s_, b)
+    ctx.run(list(range(len(bound))), fuse_combine=True)
+    ctx.check()
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        check_plan(b, op, E)
+        ref = oracle.forward(OW, op.x, op.x_scale, op.ids, op.w, round_A=oracle.ROUND_E4M3_1X128)
+        assert_close(b.y.float().cpu().numpy(), ref["y"], atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
+
+
 def test_fp8_row_counts_at_every_tile_boundary():
     """Expert row counts on and around the 128-row tile boundary of the e4m3 path (and an empty
     expert), full outputs against the mirrored oracle."""

@@ -172,6 +172,22 @@ def test_seeded_random_shapes_match_oracle(case):
         assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
+@pytest.mark.parametrize("case", [(1024, 32, 256, 128, 64, 5, 0), (600, 17, 256, 128, 300, 0, 0), (64, 8, 512, 256, 2000, 100, 2),
+                                  (64, 8, 512, 256, 2000, 100, 147), (7, 7, 256, 128, 1, 1, 0), (33, 5, 1280, 640, 777, 13, 0)],
+                         ids=["E1024_k32", "E600_k17", "one_pair", "odd_grid", "k_equals_E_one_token", "H1280_I640"])
+def test_limits_of_the_configuration_match_oracle(case):
+    """The largest expert count and top-k the library takes, k = E, a single token, a grid of one
+    CTA pair, an odd grid (single-CTA kernel), and H / I that are not powers of two."""
+    E, k, H, I, T1, T0, n_ctas = case
+    opsdef = ((synth.PREFILL, T1),) + (((synth.DECODE, T0),) if T0 else ())
+    spec = synth.Spec("lim", synth.Shape(E, k, H, I), opsdef, "zipf", 1.1, 1.0, -1.0, 7)
+    ctx, bound, ops, W = _run_spec(spec, True, budget=20, n_ctas=n_ctas)
+    OW = oracle_weights(spec, W)
+    for b, op in zip(bound, ops):
+        check_plan(b, op, E)
+        assert_close(b.y.float().cpu().numpy(), oracle.forward(OW, op.x, None, op.ids, op.w)["y"])
+
+
 def test_shared_expert_as_one_more_slot():
     """A shared (always-on) expert, Section 2.1: it is expert E-1 here, and every token carries it as
     one more top-k slot with weight 1 next to its routed experts.  The output is the routed output
