@@ -32,7 +32,12 @@ from workloads import synth  # noqa: E402
 METRIC = "moe_expert_tflops"
 UNIT = "TFLOP/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-KERNELS_PER_PLAN = 3          # histogram, scan + tile list, scatter
+def plan_kernels(n_tokens: int, top_k: int, n_experts: int) -> int:
+    """Kernels one moe_plan call launches: histogram, scan + tile list, scatter -- or one block
+    that runs all three passes when the op has at most 8192 routed rows and 256 experts."""
+    return 1 if (n_tokens * top_k <= 8192 and n_experts <= 256) else 3
+
+
 DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c2s": (20, 3), "c3s": (10, 3), "c4s": (5, 3), "c5s": (10, 3)}
 
 
@@ -181,8 +186,8 @@ class Workload:
             if self.fp8:
                 self.bytes_alg += float(active.sum()) * 3 * (sh.H // 128) * (sh.I // 128) * 4
             self.layers.append((ops, bound, host))
-        self.launches_per_step = sum(len(b) * KERNELS_PER_PLAN + 1 + (1 if self.spec.layers > 1 else 0)
-                                     for _, b, _ in self.layers)
+        self.launches_per_step = sum(sum(plan_kernels(o.T, sh.k, sh.E) for o in ops_) + 1 + (1 if self.spec.layers > 1 else 0)
+                                     for ops_, _, _ in self.layers)
 
     def step(self, ev=None):
         """Whole hot path for one batch; ev (optional) collects (before_run, after_run) events."""
@@ -445,7 +450,8 @@ def persistent_layers(w: Workload, steps: int, warmup: int):
     same = all(torch.equal(b.y, bo.y) for b, (_, b_old, _) in zip([bound[i:i + 2] for i in range(0, len(bound), 2)], w.layers)
                for b, bo in zip(b, b_old)) if all(len(x[1]) == 2 for x in w.layers) else None
     return {"ms_per_step": ms, "value": w.flops / (ms / 1e3) / 1e12, "unit": UNIT, "ops_in_launch": len(bound),
-            "launches_per_step": len(bound) * KERNELS_PER_PLAN + 1, "outputs_equal_per_layer_launches": same,
+            "launches_per_step": sum(plan_kernels(o.T, sh.k, sh.E) for ops_, _, _ in w.layers for o in ops_) + 1,
+            "outputs_equal_per_layer_launches": same,
             "per_layer_launches_ms_per_step_alternating": float(np.mean(t_per))}
 
 

@@ -15,6 +15,7 @@ cudaError_t launch_combine(const OpDev* d_op, int T, int k, int H, cudaStream_t 
 cudaError_t prepare_run_kernel();
 cudaError_t launch_run(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream);
 cudaError_t prepare_pair_kernel();
+cudaError_t prepare_plan_kernels();
 cudaError_t launch_pair(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream);
 }  // namespace moe
 
@@ -182,7 +183,9 @@ int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_c
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
       qres != cudaDriverEntryPointSuccess || !fn)
     return MOE_ECUDA;
-  if (prepare_run_kernel() != cudaSuccess || prepare_pair_kernel() != cudaSuccess) return MOE_ECUDA;
+  if (prepare_run_kernel() != cudaSuccess || prepare_pair_kernel() != cudaSuccess ||
+      prepare_plan_kernels() != cudaSuccess)
+    return MOE_ECUDA;
   moe_ctx* ctx = new (std::nothrow) moe_ctx();
   if (!ctx) return MOE_ENOSPC;
   ctx->cfg = *cfg;

@@ -15,12 +15,9 @@ constexpr int kPlanThreads = 256;
 constexpr int kPlanWarps = kPlanThreads / 32;
 
 // ---------------------------------------------------------------- K1: per-warp histograms
-__global__ void __launch_bounds__(kPlanThreads)
-plan_hist_kernel(const OpDev* __restrict__ op, Global* g, int slot, int R, int E) {
-  extern __shared__ int sm[];                 // [kPlanWarps][E]
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int chunk = blockIdx.x * kPlanWarps + warp;
-  int* h = sm + warp * E;
+// one warp, one chunk of kPlanChunk routed rows; h: the warp's E counters in shared memory
+__device__ __forceinline__ void hist_chunk(const OpDev* __restrict__ op, Global* g, int slot, int R, int E,
+                                           int chunk, int* h, int lane) {
   for (int e = lane; e < E; e += 32) h[e] = 0;
   __syncwarp();
   const int* ids = op->topk_ids;
@@ -46,6 +43,13 @@ plan_hist_kernel(const OpDev* __restrict__ op, Global* g, int slot, int R, int E
   int* out = op->plan_hist + (size_t)chunk * E;
   if (base < R)
     for (int e = lane; e < E; e += 32) out[e] = h[e];
+}
+
+__global__ void __launch_bounds__(kPlanThreads)
+plan_hist_kernel(const OpDev* __restrict__ op, Global* g, int slot, int R, int E) {
+  extern __shared__ int sm[];                 // [kPlanWarps][E]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  hist_chunk(op, g, slot, R, E, blockIdx.x * kPlanWarps + warp, sm + warp * E, lane);
 }
 
 // exclusive scan of one int per thread over a 1024-thread block
@@ -78,9 +82,9 @@ __device__ inline int block_excl_scan(int v, int* total, int* warp_sums) {
 }
 
 // ---------------------------------------------------------------- K2: scans + tile table + tile list
-__global__ void __launch_bounds__(1024)
-plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int NT1, int NT2,
-                 int T, int work_rows) {
+// the whole block of 1024 threads
+__device__ __forceinline__ void scan_body(const OpDev* __restrict__ op, int n_chunks, int R, int E, int NT1, int NT2,
+                                          int T, int work_rows) {
   __shared__ int warp_sums[33];
   __shared__ int s_cnt[kMaxExperts], s_grp[kMaxExperts], s_moff[kMaxExperts], s_off[kMaxExperts];
   __shared__ int s_part[1024];
@@ -92,8 +96,8 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   // column sums of the per-warp histograms, the device prefix sum over experts, then the base
   // rank of every (warp chunk, expert).  Reads and writes use different arrays so that the
   // loads of a column do not wait on the stores.
-  const int* __restrict__ hist = op->plan_hist;
-  int* __restrict__ base = op->plan_base;
+  const int* hist = op->plan_hist;        // no __restrict__: the one-block plan wrote it earlier in the same kernel
+  int* base = op->plan_base;
   // the 1024 threads split every expert's column into `parts` chunk ranges
   const int parts = max(1, 1024 / E);
   const int part = threadIdx.x / E, pe = threadIdx.x % E;
@@ -212,15 +216,17 @@ plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int N
   }
 }
 
+__global__ void __launch_bounds__(1024)
+plan_scan_kernel(const OpDev* __restrict__ op, int n_chunks, int R, int E, int NT1, int NT2,
+                 int T, int work_rows) {
+  scan_body(op, n_chunks, R, E, NT1, NT2, T, work_rows);
+}
+
 // ---------------------------------------------------------------- K3: stable scatter
-__global__ void __launch_bounds__(kPlanThreads)
-plan_scatter_kernel(const OpDev* __restrict__ op, int R, int E) {
-  extern __shared__ int sm[];                 // [kPlanWarps][E] running rank per expert
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int chunk = blockIdx.x * kPlanWarps + warp;
+// one warp, one chunk; run: the warp's E running ranks in shared memory
+__device__ __forceinline__ void scatter_chunk(const OpDev* __restrict__ op, int R, int E, int chunk, int* run, int lane) {
   const int base = chunk * kPlanChunk;
   if (base >= R) return;
-  int* run = sm + warp * E;
   const int* src = op->plan_base + (size_t)chunk * E;
   for (int e = lane; e < E; e += 32) run[e] = src[e];
   __syncwarp();
@@ -237,7 +243,7 @@ plan_scatter_kernel(const OpDev* __restrict__ op, int R, int E) {
   for (int it = 0; it < kPlanChunk / 32; ++it) {
     const int i = base + it * 32 + lane;
     int id = my[it];
-    if (id < 0 || id >= E) id = -1;         // reported by the histogram kernel
+    if (id < 0 || id >= E) id = -1;         // reported by the histogram pass
     const unsigned peers = __match_any_sync(0xffffffffu, id);
     const unsigned before = peers & ((1u << lane) - 1);
     int p = -1;
@@ -252,12 +258,50 @@ plan_scatter_kernel(const OpDev* __restrict__ op, int R, int E) {
   }
 }
 
+__global__ void __launch_bounds__(kPlanThreads)
+plan_scatter_kernel(const OpDev* __restrict__ op, int R, int E) {
+  extern __shared__ int sm[];                 // [kPlanWarps][E] running rank per expert
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  scatter_chunk(op, R, E, blockIdx.x * kPlanWarps + warp, sm + warp * E, lane);
+}
+
+// ---------------------------------------------------------------- small ops: the three passes in one block
+// An op of at most kSmallChunks chunks (a decode batch) is planned by ONE block of 32 warps: the
+// histogram scratch written by the first pass is read back by the same block, so two launches and
+// their gaps go away (they are about half of a small plan's time).
+constexpr int kSmallChunks = 32;
+constexpr int kSmallMaxExperts = 256;
+
+__global__ void __launch_bounds__(1024)
+plan_small_kernel(const OpDev* __restrict__ op, Global* g, int slot, int n_chunks, int R, int E, int NT1, int NT2,
+                  int T, int work_rows) {
+  extern __shared__ int sm[];                 // [32 warps][E]
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  if (warp < n_chunks) hist_chunk(op, g, slot, R, E, warp, sm + warp * E, lane);
+  __threadfence_block();
+  __syncthreads();
+  scan_body(op, n_chunks, R, E, NT1, NT2, T, work_rows);
+  __threadfence_block();
+  __syncthreads();
+  if (warp < n_chunks) scatter_chunk(op, R, E, warp, sm + warp * E, lane);
+}
+
+cudaError_t prepare_plan_kernels() {
+  return cudaFuncSetAttribute(plan_small_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              kSmallChunks * kSmallMaxExperts * (int)sizeof(int));
+}
+
 cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, int E, int NT1,
                         int NT2, int work_rows, cudaStream_t stream) {
   const int R = T * k;
   const int n_chunks = (R + kPlanChunk - 1) / kPlanChunk;
   const int blocks = (n_chunks + kPlanWarps - 1) / kPlanWarps;
   const size_t smem = (size_t)kPlanWarps * E * sizeof(int);
+  if (n_chunks <= kSmallChunks && E <= kSmallMaxExperts) {
+    plan_small_kernel<<<1, 1024, (size_t)kSmallChunks * E * sizeof(int), stream>>>(d_op, g, slot, n_chunks, R, E, NT1, NT2, T,
+                                                                                 work_rows);
+    return cudaGetLastError();
+  }
   if (blocks > 0) plan_hist_kernel<<<blocks, kPlanThreads, smem, stream>>>(d_op, g, slot, R, E);
   plan_scan_kernel<<<1, 1024, 0, stream>>>(d_op, n_chunks, R, E, NT1, NT2, T, work_rows);
   if (blocks > 0) plan_scatter_kernel<<<blocks, kPlanThreads, smem, stream>>>(d_op, R, E);
