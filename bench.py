@@ -349,8 +349,6 @@ def tile_stats(w: Workload):
     w.step()
     w.ctx.check()
     log = w.ctx.tile_log()
-    if os.environ.get("MOE_BENCH_DUMP_LOG"):
-        np.save(os.environ["MOE_BENCH_DUMP_LOG"], log)
     out = {"corun": _log_summary(log)}
     _, bound, _ = w.layers[-1]
     dec = [s for s, b in enumerate(bound) if b.c.cls == 0]

@@ -122,7 +122,13 @@ void moe_destroy(moe_ctx_t* ctx);
  * packed per-expert layout of Section 2.4), and the op's tile table, whose length is
  * the footprint x_moe = sum_{e: m_e>0} ceil(m_e / M_t) of Section 6.2.  Binds `op` to
  * `slot`; the struct is copied, the buffers it names must stay valid until the work
- * enqueued on them has finished. */
+ * enqueued on them has finished.
+ * An expert id outside [0, n_experts) is recorded as MOE_EBADID (detail: slot, flat
+ * index, id).  Such a row gets no packed position: flat_to_sorted[i] = -1, the unclaimed
+ * tail of sorted_to_flat is -1, counts and offsets cover the accepted rows only, and the
+ * slot is left without a plan -- moe_run and moe_combine enqueued behind it do nothing for
+ * it, and once moe_status has returned the error they answer MOE_ENOTPLANNED until the
+ * slot is planned again. */
 int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
 
 /* The persistent expert kernel over the planned ops in `slots` (one launch): every CTA
@@ -134,11 +140,19 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
  * only between tiles (Section 4.2), so results do not depend on the schedule.
  * Ops of one class are served in the order given.  With fuse_combine != 0 the
  * router-weighted combine runs as tiles of the same launch and y is final when the
- * kernel ends; otherwise call moe_combine. */
+ * kernel ends; otherwise call moe_combine.
+ * An op without tokens has no tiles: it counts as finished as soon as the op it comes
+ * after has (at once if there is none), its done and notify words are set then, and its
+ * ready word is not consulted.
+ * `ready`, `done` and `notify` words may also live in pinned host memory that the device
+ * can address (they are read and written at system scope), so the host can make an op
+ * ready, or learn of progress, while the kernel runs; every device-side wait on them is
+ * bounded by wait_limit_us. */
 int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, void* stream);
 
 /* Post-processing: y[t,:] = sum_j w[t,j] * D[flat_to_sorted[t*k+j],:], slots added in
- * order j = 0..k-1 in fp32 (Section 2.1, "combines their outputs"). */
+ * order j = 0..k-1 in fp32 (the last step of the MoE module of Section 2.1).  A permutation
+ * entry outside [0, T*k) is reported as MOE_EBOUNDS and contributes nothing. */
 int moe_combine(moe_ctx_t* ctx, int slot, void* stream);
 
 /* Decode SM budget q of Section 6.4: a stream-ordered 4-byte write to the device word
@@ -185,6 +199,8 @@ int moe_read_tile_log(moe_ctx_t* ctx, moe_tile_rec_t* host_out, int max_records,
  *   - limits: n_tokens * top_k <= MOE_PLAN_STATIC_MAX_ROWS and n_experts <=
  *     MOE_PLAN_STATIC_MAX_EXPERTS, else MOE_ENOSPC (nothing is launched);
  *   - all pointers are device pointers owned by the caller, sizes as in moe_op_t;
+ *   - `stream` must belong to the device that is current when the call is made: the
+ *     scratch array's address is looked up on the current device;
  *   - expert ids outside [0, n_experts) are skipped silently (moe_plan reports them);
  *   - every call looks up the scratch array's device address (nothing is cached, so a device
  *     reset between calls is harmless); the first look-up on a device may load the library's

@@ -27,20 +27,6 @@ def stale() -> bool:
     return any(os.path.getmtime(d) > t for d in deps)
 
 
-def build_probe(verbose: bool = False) -> str:
-    """The same library with the in-kernel timers compiled in (-DMOE_TIMING_PROBE): the MMA, producer
-    and epilogue warps of one CTA record clock64 stamps per k-block into the tile-log area, which
-    moe_read_tile_log then returns as raw 64-bit words (the log itself is off in this build).  For
-    kernel studies only; never loaded by the package."""
-    out = os.path.join(HERE, "libmoe_apk_probe.so")
-    res = subprocess.run([NVCC] + FLAGS + ["-DMOE_TIMING_PROBE", "-o", out] + sources(), capture_output=True, text=True)
-    if verbose or res.returncode != 0:
-        print(res.stdout + res.stderr)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed")
-    return out
-
-
 def build(force: bool = False, verbose: bool = False) -> str:
     if force or stale():
         cmd = [NVCC] + FLAGS + ["-o", LIB] + sources()
@@ -53,8 +39,4 @@ def build(force: bool = False, verbose: bool = False) -> str:
 
 
 if __name__ == "__main__":
-    import sys
-    if "--probe" in sys.argv:
-        print(build_probe(verbose=True))
-    else:
-        build(force=True, verbose=True)
+    build(force=True, verbose=True)

@@ -8,6 +8,7 @@ constexpr int kCombTokensPerBlock = 4;
 
 __global__ void __launch_bounds__(kCombThreads)
 combine_kernel(const OpDev* __restrict__ op, int T, int k, int H) {
+  if (op->plan->planned == 0) return;          // the slot's plan was rejected: there is no permutation to follow
   const int t0 = blockIdx.x * kCombTokensPerBlock;
   const int t1 = min(T, t0 + kCombTokensPerBlock);
   if (t0 < t1) combine_tokens(op, t0, t1, k, H, threadIdx.x, kCombThreads);

@@ -1,7 +1,9 @@
 // Router-weighted combine (post-processing): y[t,:] = sum_j w[t,j] * D[flat_to_sorted[t*k+j],:]
-// with the k slots added in order in fp32 (Section 2.1 of the paper: the module "combines
-// their outputs").  One device routine serves the stand-alone kernel and the combine tiles
-// of the persistent kernel.
+// with the k slots added in order in fp32 (the last step of the MoE module of Section 2.1 of the
+// paper).  One device routine serves the stand-alone kernel and the combine tiles of the
+// persistent kernel.  A permutation entry outside [0, T*k) -- left by a plan that rejected an
+// expert id -- is reported as MOE_EBOUNDS and its slot contributes nothing; no address is formed
+// from it.
 #pragma once
 #include "moe_dev.cuh"
 
@@ -29,8 +31,14 @@ __device__ __forceinline__ void combine_add4(float (&acc)[8], const uint4 (&d)[4
   }
 }
 
+__device__ __forceinline__ int f2s_entry(const OpDev* op, int i) { return op->flat_to_sorted[i]; }
+
 __device__ __noinline__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, int H, int tid,
-                                      int nthr) {
+                                                   int nthr) {
+  const unsigned n_rows = (unsigned)op->n_rows;
+  // every permutation entry of these tokens is checked once, ahead of the loops that use them
+  for (int i = t0 * k + tid; i < t1 * k; i += nthr)
+    if ((unsigned)f2s_entry(op, i) >= n_rows) report(op->status, MOE_EBOUNDS, i / k, i % k, f2s_entry(op, i), 2);
   const int vec_per_row = H / 8;
   const uint4* D = reinterpret_cast<const uint4*>(op->D);
   uint4* y = reinterpret_cast<uint4*>(op->y);
@@ -53,8 +61,10 @@ __device__ __noinline__ inline void combine_tokens(const OpDev* op, int t0, int 
         off[i] = 0u;
         wj[i] = 0.f;
         if (i < k) {
-          off[i] = (unsigned)f2s[(size_t)t * k + i] * (unsigned)vec_per_row;
-          wj[i] = w[(size_t)t * k + i];
+          const unsigned p = (unsigned)f2s[(size_t)t * k + i];
+          const bool ok = p < n_rows;                      // reported by the check above; adds nothing
+          off[i] = ok ? p * (unsigned)vec_per_row : 0u;
+          wj[i] = ok ? w[(size_t)t * k + i] : 0.f;
         }
       }
       const uint4* src = D + sub;
@@ -107,8 +117,10 @@ __device__ __noinline__ inline void combine_tokens(const OpDev* op, int t0, int 
         d[i] = make_uint4(0u, 0u, 0u, 0u);
         if (j < k) {
           const int p = f2s[(size_t)t * k + j];
-          wj[i] = w[(size_t)t * k + j];
-          d[i] = D[(size_t)p * vec_per_row + v];
+          if ((unsigned)p < n_rows) {
+            wj[i] = w[(size_t)t * k + j];
+            d[i] = D[(size_t)p * vec_per_row + v];
+          }
         }
       }
 #pragma unroll

@@ -45,7 +45,7 @@ struct PlanState {
   int n_mtiles;       // x_moe
   int n_gemm_tiles;   // queue entries of kind gate/up or down
   int n_comb_tiles;   // queue entries of kind combine (follow the GEMM entries)
-  int planned;        // 1 after moe_plan
+  int planned;        // 1 after a moe_plan that accepted every expert id, else 0
 };
 
 // Zeroed by moe_run before every launch.
@@ -55,6 +55,8 @@ struct RunState {
   int done;           // 1 when the op has fully finished
   int pad;
 };
+
+struct Status;
 
 struct __align__(128) OpDev {
   CUtensorMap tm_a8;    // [Rmax, I]   box {64, 8}   packed intermediate, 8 consecutive rows
@@ -94,6 +96,7 @@ struct __align__(128) OpDev {
   PlanState* plan;
   RunState* run;
   int* g1_done;          // [max_mtiles] committed gate/up tiles per work tile
+  Status* status;        // the context's device status block
 };
 
 struct Status {   // first error wins (atomicCAS on code)
@@ -126,14 +129,11 @@ struct RunArgs {
   int fuse_combine;
   int E, k, H, I;
   int dtype, kb_elems;    // MOE_DTYPE_*; K elements per pipeline stage (64 bf16 / 128 e4m3)
-#ifdef MOE_TIMING_PROBE
-  long long* dbg;
-#endif
   long long wait_ns;
   int slots[kMaxOps];
 };
 
-__device__ inline void report(Status* st, int code, int d0, int d1, int d2, int d3) {
+__device__ __noinline__ inline void report(Status* st, int code, int d0, int d1, int d2, int d3) {
   if (atomicCAS(&st->code, 0, code) == 0) {
     st->detail[0] = d0; st->detail[1] = d1; st->detail[2] = d2; st->detail[3] = d3;
   }

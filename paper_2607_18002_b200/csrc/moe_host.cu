@@ -41,6 +41,8 @@ int check_config(const moe_config_t* c) {
   if (c->top_k < 1 || c->top_k > 32 || c->top_k > c->n_experts) return MOE_EINVAL;
   if (c->hidden < kTileN2 || c->hidden % kTileN2) return MOE_EINVAL;
   if (c->inter < kTileN1 || c->inter % kTileN1) return MOE_EINVAL;
+  // a queue entry keeps its n-tile index in eight bits
+  if (c->inter / kTileN1 > 255 || c->hidden / kTileN2 > 255) return MOE_EINVAL;
   if (c->dtype != MOE_DTYPE_BF16 && c->dtype != MOE_DTYPE_FP8_E4M3) return MOE_EINVAL;
   if (c->max_tokens_per_op < 1 || c->max_ops < 1 || c->max_ops > kMaxOps) return MOE_EINVAL;
   if ((long long)c->max_tokens_per_op * c->top_k > (1 << 20) * (long long)kTileM) return MOE_EINVAL;
@@ -259,6 +261,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   h.plan = reinterpret_cast<PlanState*>(sb + L.plan_off);
   h.run = reinterpret_cast<RunState*>(ctx->rs_base(slot));
   h.g1_done = reinterpret_cast<int*>(ctx->rs_base(slot) + sizeof(RunState));
+  h.status = &ctx->g()->status;
   // Re-planning a slot with the same buffers (the usual serving loop) reuses the descriptors
   // already on the device: encoding seven tensor maps and uploading them is host time.
   const bool same = ctx->uploaded[slot] && memcmp(&ctx->ops[slot], op, sizeof(moe_op_t)) == 0;
@@ -275,15 +278,18 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
       if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
       if (rc) return rc;
     }
+    ctx->planned[slot] = false;
     write_op_kernel<<<1, 128, 0, st>>>(h, ctx->op_dev(slot));
-    if (cudaGetLastError() != cudaSuccess) return MOE_ECUDA;
+    if (cudaGetLastError() != cudaSuccess) { ctx->uploaded[slot] = false; return MOE_ECUDA; }
     ctx->host_ops[slot] = h;
+    ctx->ops[slot] = *op;             // what the device copy of the slot now describes
     ctx->uploaded[slot] = true;
   }
   if (launch_plan(ctx->op_dev(slot), ctx->g(), slot, op->n_tokens, c.top_k, c.n_experts, L.NT1, L.NT2,
-                  c.dtype == MOE_DTYPE_FP8_E4M3 ? kWorkRowsFp8 : kWorkRowsBf16, st) != cudaSuccess)
+                  c.dtype == MOE_DTYPE_FP8_E4M3 ? kWorkRowsFp8 : kWorkRowsBf16, st) != cudaSuccess) {
+    ctx->planned[slot] = false;
     return MOE_ECUDA;
-  ctx->ops[slot] = *op;
+  }
   ctx->planned[slot] = true;
   return MOE_OK;
 }
@@ -317,10 +323,6 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
   a.dtype = c.dtype;
   a.kb_elems = c.dtype == MOE_DTYPE_FP8_E4M3 ? 128 : kBlockK;
   a.wait_ns = (long long)c.wait_limit_us * 1000;
-#ifdef MOE_TIMING_PROBE
-  a.dbg = reinterpret_cast<long long*>(ctx->ws + ctx->L.log_off);   // the tile log area doubles as probe buffer
-  a.log_cap = 0;
-#endif
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
   const cudaError_t le = ctx->pair_kernel ? launch_pair(a, ctx->rh(), ctx->n_ctas, st)
@@ -374,6 +376,8 @@ int moe_status(moe_ctx_t* ctx, int32_t* code, int32_t detail[4]) {
   if (cudaMemcpy(&s, &ctx->g()->status, sizeof(s), cudaMemcpyDeviceToHost) != cudaSuccess) return MOE_ECUDA;
   *code = s.code;
   if (detail) for (int i = 0; i < 4; ++i) detail[i] = s.detail[i];
+  // a plan that met an expert id out of range left its slot without a usable permutation
+  if (s.code == MOE_EBADID && s.detail[0] >= 0 && s.detail[0] < ctx->cfg.max_ops) ctx->planned[s.detail[0]] = false;
   if (s.code != 0 || s.abort != 0)
     if (cudaMemset(&ctx->g()->status, 0, sizeof(Status)) != cudaSuccess) return MOE_ECUDA;
   return MOE_OK;
@@ -405,9 +409,6 @@ int moe_read_tile_log(moe_ctx_t* ctx, moe_tile_rec_t* host_out, int max_records,
   RunHead rh;
   if (cudaMemcpy(&rh, ctx->rh(), sizeof(rh), cudaMemcpyDeviceToHost) != cudaSuccess) return MOE_ECUDA;
   int cnt = (int)rh.log_count;
-#ifdef MOE_TIMING_PROBE
-  cnt = ctx->cfg.tile_log_entries;
-#endif
   if (cnt > ctx->cfg.tile_log_entries) cnt = ctx->cfg.tile_log_entries;
   if (cnt > max_records) cnt = max_records;
   if (cnt > 0 && cudaMemcpy(host_out, ctx->ws + ctx->L.log_off, (size_t)cnt * sizeof(moe_tile_rec_t),

@@ -122,6 +122,9 @@ __device__ __forceinline__ void scan_body(const OpDev* __restrict__ op, int n_ch
     s_off[e] = off;
   }
   if (e == 0) op->offsets[E] = total;
+  // rows with a rejected expert id take no packed position: the tail of the permutation that no row
+  // will claim is marked, so that nothing downstream mistakes stale memory for an index
+  for (int p = total + (int)threadIdx.x; p < R; p += (int)blockDim.x) op->sorted_to_flat[p] = -1;
   __syncthreads();
   if (part < parts) {
     int run = s_off[pe];
@@ -211,7 +214,7 @@ __device__ __forceinline__ void scan_body(const OpDev* __restrict__ op, int n_ch
     ps.n_mtiles = x_moe;
     ps.n_gemm_tiles = n_gemm;
     ps.n_comb_tiles = n_comb;
-    ps.planned = 1;
+    ps.planned = total == R ? 1 : 0;        // a plan with a rejected id leaves the slot without tiles to run
     *op->plan = ps;
   }
 }
@@ -254,6 +257,8 @@ __device__ __forceinline__ void scatter_chunk(const OpDev* __restrict__ op, int 
     if (p >= 0 && p < R) {
       s2f[p] = i;
       f2s[i] = p;
+    } else if (i < R) {
+      f2s[i] = -1;                          // a rejected id: the row has no packed position
     }
   }
 }

@@ -1,7 +1,7 @@
 // moe_route: the router ahead of the plan step -- per token the k experts with the largest logits
-// and the router weights softmax(logits) renormalised over those k (Section 2.1 of the paper: "a
-// router selects the top-k routed experts for each token"; the paper does not fix the arithmetic,
-// this is the softmax -> top-k -> renormalise form of the seeded workloads).
+// and the router weights softmax(logits) renormalised over those k (the router step of the MoE
+// module of Section 2.1 of the paper; the paper does not fix the arithmetic, this is the
+// softmax -> top-k -> renormalise form of the seeded workloads).
 //
 // One warp per token.  Each lane holds the logits e = lane, lane + 32, ... in registers (E <= 1024);
 // k rounds of a warp arg-max pick the experts in order of decreasing logit, ties to the lower

@@ -56,10 +56,6 @@ struct SharedCtl {
   unsigned tmem_base;
   alignas(16) unsigned char epi_scratch[8][2048];   // per epilogue warp: 32 rows x 64 bytes
   QueueTables qt;
-#ifdef MOE_TIMING_PROBE
-  int dbg_e;
-  int dbg_w[8];
-#endif
 };
 
 constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + sizeof(SharedCtl);
@@ -88,7 +84,12 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
   const float* sx;
   const float *sw0, *sw1;
   if (g1) {
-    const int tok = valid ? op->sorted_to_flat[ti.row0 + row] / a.k : 0;
+    int tok = 0;
+    if (valid) {
+      const int flat = op->sorted_to_flat[ti.row0 + row];
+      if ((unsigned)flat < (unsigned)op->n_rows) tok = flat / a.k;
+      else report(c.st, MOE_EBOUNDS, ti.slot, ti.row0 + row, flat, 1);
+    }
     sx = op->x_scale + (size_t)tok * HB;
     sw0 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + ti.n) * HB;
     sw1 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + IB + ti.n) * HB;
@@ -119,15 +120,9 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
     const float s0 = nfx * nw0, s1 = nfx * nw1;
     if (kb + 1 < ti.kblocks) { nfx = sx[kb + 1]; nw0 = sw0[kb + 1]; nw1 = sw1[kb + 1]; }
     const int pb = kb & 1;
-#ifdef MOE_TIMING_PROBE
-    const long long e0 = clock64();
-#endif
     if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->pfull[pb], (eph >> pb) & 1u, 19))) return false;
     eph ^= 1u << pb;
     tc_fence_after();
-#ifdef MOE_TIMING_PROBE
-    const long long e1 = clock64();
-#endif
     // eight 16-column chunks (four per half); the load of chunk c+1 is in flight while chunk c
     // is multiplied in
     const unsigned pbase = lane_addr + (unsigned)(pb * 256 + ch * 64);
@@ -145,12 +140,6 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
     tc_fence_before();
     __syncwarp();                                 // every lane's TMEM loads have completed
     if (lane == 0) mbar_arrive(&sc->pempty[pb]); // one arrival per warp: the partial buffer may be overwritten
-#ifdef MOE_TIMING_PROBE
-    if (blockIdx.x == 7 && lane == 0 && sc->dbg_w[warp - 8] < 2048) {
-      long long* pp = a.dbg + 16384 + (size_t)(warp - 8) * 8192 + (size_t)sc->dbg_w[warp - 8]++ * 4;
-      pp[0] = e0; pp[1] = e1; pp[2] = clock64(); pp[3] = ti.kind * 1000 + kb;
-    }
-#endif
   }
   // the accumulator is complete
   if (g1) {
@@ -235,10 +224,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
   Ctx c{&args, &args.g->status};
 
   if (threadIdx.x == 0) {
-#ifdef MOE_TIMING_PROBE
-    sc->dbg_e = 0;
-    for (int i = 0; i < 8; ++i) sc->dbg_w[i] = 0;
-#endif
     for (int s = 0; s < kNS; ++s) {
       mbar_init(&sc->full[s], 1);
       mbar_init(&sc->fullA[s], kGatherThreads);
@@ -260,6 +245,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       mbar_init(&sc->done[s], 256);
     }
     build_queues(&args, &sc->qt);
+    if (blockIdx.x == 0) finish_empty_ops(&args, -1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_proxy();
   }
@@ -287,9 +273,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     // kClaimAt-th k-block), so the claim's round trips and the first loads of the next tile
     // overlap the current tile's tail instead of draining the pipeline.  A CTA therefore
     // holds at most one claimed tile beyond the one it is executing.
-#ifdef MOE_TIMING_PROBE
-    int dbg_i = 0;
-#endif
     int stage = 0, islot = 0;
     unsigned ph = 0, iph = 0;
     TileInfo ti, nx;
@@ -387,9 +370,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
   } else if (warp == 1) {
     MOE_REGS_DEC();
     // ============================================================ MMA issuer
-#ifdef MOE_TIMING_PROBE
-    int dbg_i = 0, dbg_t = 0;
-#endif
     int stage = 0, islot = 0;
     unsigned ph = 0, iph = 0, aph[2] = {0, 0}, pph = 0;
     AccUse accs;
@@ -400,38 +380,19 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       const int rows = sc->info[islot].rows;
       if (kind == kEnd) break;
       bool fail = false;
-#ifdef MOE_TIMING_PROBE
-      const long long tt0 = clock64();
-      long long tt1 = 0, tt2 = 0;
-#endif
       if (kFp8 && kind != kCombine) {
         // FP8 with fp32 block scales: the tensor core cannot apply a scale per 128-deep K block,
         // so every k-block (= one scale block) is multiplied into a FRESH partial buffer, one
         // per 128-column half of the weight tile (each half has a single weight scale), and the
         // epilogue warps scale-and-add it into the fp32 accumulator columns of TMEM.
         for (int kb = 0; kb < kblocks; ++kb) {
-#ifdef MOE_TIMING_PROBE
-          const long long q0 = clock64();
-#endif
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
-#ifdef MOE_TIMING_PROBE
-          const long long q1 = clock64();
-#endif
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], ph, 12))) { fail = true; break; }
-#ifdef MOE_TIMING_PROBE
-          const long long q2 = clock64();
-#endif
           {
             const int pb = kb & 1;                        // partial buffer of this k-block
             if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->pempty[pb], ((pph >> pb) & 1u) ^ 1u, 18))) { fail = true; break; }
             pph ^= 1u << pb;
             tc_fence_after();
-#ifdef MOE_TIMING_PROBE
-            if (blockIdx.x == 7 && lane == 0 && dbg_i < 4096) {
-              long long* pp = args.dbg + (size_t)dbg_i++ * 4;
-              pp[0] = q0; pp[1] = q1; pp[2] = q2; pp[3] = clock64();
-            }
-#endif
             {
               fence_async_proxy_smem();
               const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
@@ -455,24 +416,15 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         if (use0 && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[0], aph[0] ^ 1u, 7))) break;
         if (use1 && !pair && !__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[1], aph[1] ^ 1u, 7))) break;
         tc_fence_after();
-#ifdef MOE_TIMING_PROBE
-        tt1 = clock64();
-#endif
         const unsigned d0 = tmem + (use0 ? 0u : (unsigned)kAccCols);     // accumulator of rows 0..127
         for (int kb = 0; kb < kblocks; ++kb) {
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->full[stage], ph, 8))) { fail = true; break; }
-#ifdef MOE_TIMING_PROBE
-          const long long t_fullB = clock64();
-#endif
           // The gather warps arrive on fullA for every k-block (with the copied rows of a
           // gate/up tile, empty-handed otherwise): being part of every stage hand-off keeps them
           // within one phase of the stage barriers they wait on.
           if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->fullA[stage], ph, 12))) { fail = true; break; }
           tc_fence_after();
           if (lane == 0) {
-#ifdef MOE_TIMING_PROBE
-            if (blockIdx.x == 7 && dbg_i < 4096) { args.dbg[dbg_i * 4 + 1] = clock64(); args.dbg[dbg_i * 4 + 2] = kind * 1000 + rows; }
-#endif
             fence_async_proxy_smem();                    // cp.async-written rows -> tensor core reads
             const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
             const unsigned long long ad = umma_desc(sA, kRowBytes), bd = umma_desc(sA + kBOff, kRowBytes);
@@ -483,9 +435,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           if (pair && kb == 0) {                         // accumulator 1 is needed from here on
             if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->tempty[1], aph[1] ^ 1u, 7))) { fail = true; break; }
             tc_fence_after();
-#ifdef MOE_TIMING_PROBE
-            tt2 = clock64();
-#endif
           }
           if (lane == 0) {
             const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
@@ -497,9 +446,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
                 tc_mma_bf16(tmem + (unsigned)kAccCols, ad1 + 2ull * k4, bd + 2ull * k4, kIdesc, (kb | k4) ? 1u : 0u);
             }
             tc_commit(&sc->empty[stage]);               // frees the stage when the MMAs retire
-#ifdef MOE_TIMING_PROBE
-            if (blockIdx.x == 7 && dbg_i < 4096) args.dbg[dbg_i++ * 4 + 3] = t_fullB;
-#endif
           }
           __syncwarp();
           if (++stage == kNS) { stage = 0; ph ^= 1u; }
@@ -508,12 +454,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         if (lane == 0) {                                 // accumulator(s) complete
           if (use0) tc_commit(&sc->tfull[0]);
           if (use1) tc_commit(&sc->tfull[1]);
-#ifdef MOE_TIMING_PROBE
-          if (blockIdx.x == 7 && dbg_t < 512) {
-            long long* pp = args.dbg + 8192 * 4 + (size_t)dbg_t++ * 8;
-            pp[0] = tt0; pp[1] = tt1; pp[2] = tt2; pp[3] = clock64(); pp[4] = kind * 1000 + rows;
-          }
-#endif
         }
         __syncwarp();
         if (use0) aph[0] ^= 1u;
@@ -559,11 +499,17 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       const unsigned char* X = static_cast<const unsigned char*>(op->x) + chunk * 16;
       const size_t pitch = (size_t)args.H * kEl;
       int tok[kPasses];
+      const int n_rows = op->n_rows;
+      bool bad = false;
 #pragma unroll
       for (int j = 0; j < kPasses; ++j) {
         const int r = rbase + kRowsPerPass * j;
-        tok[j] = r < rows ? op->sorted_to_flat[row0 + r] / args.k : -1;
+        const int flat = r < rows ? op->sorted_to_flat[row0 + r] : 0;
+        const bool in_range = (unsigned)flat < (unsigned)n_rows;    // an index the plan never wrote is reported
+        bad |= !in_range;                                            // below and its row is skipped
+        tok[j] = (r < rows && in_range) ? flat / args.k : -1;
       }
+      if (bad) report(c.st, MOE_EBOUNDS, slot, row0, rows, 0);
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
         const int stage = (int)(kiter % kNS);
@@ -615,9 +561,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
     int islot = 0;
     unsigned iph = 0, aph[2] = {0, 0}, eph = 0, xph = 0;
     AccUse accs;
-#ifdef MOE_TIMING_PROBE
-    int dbg_e = 0;
-#endif
     unsigned char* scratch = sc->epi_scratch[warp - 8];
     const int srow = lane >> 2, schunk = lane & 3;          // this lane's part of a store
     while (true) {
@@ -640,16 +583,10 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
 #pragma unroll
         for (int b = 0; b < 2; ++b) {
           if (!use[b]) continue;
-#ifdef MOE_TIMING_PROBE
-          const long long te0 = clock64();
-#endif
           ok = __all_sync(0xffffffffu, mbar_wait_inline(c, &sc->tfull[b], aph[b], 10));
           if (!ok) break;
           aph[b] ^= 1u;
           tc_fence_after();
-#ifdef MOE_TIMING_PROBE
-          const long long te1 = clock64();
-#endif
           const int rbase = pair ? b * kTileM : 0;               // first tile row of this accumulator
           const int nrows = min(ti.rows - rbase, kTileM);
           if (q * 32 < nrows) {
@@ -704,12 +641,6 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           }
           tc_fence_before();
           mbar_arrive(&sc->tempty[b]);            // accumulator may be overwritten
-#ifdef MOE_TIMING_PROBE
-          if (blockIdx.x == 7 && warp == 8 && lane == 0 && dbg_e < 1024) {
-            long long* pp = args.dbg + 12288 * 4 + (size_t)sc->dbg_e++ * 4;
-            pp[0] = te0; pp[1] = te1; pp[2] = clock64(); pp[3] = ti.kind * 1000 + ti.rows + b * 100000;
-          }
-#endif
         }
       }
       if (!ok) break;

@@ -231,6 +231,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       mbar_init(&sc->taken[s], 1);
     }
     if (leader) build_queues(&args, &sc->qt);
+    if (blockIdx.x == 0) finish_empty_ops(&args, -1);
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     fence_async_proxy();
   }
@@ -287,9 +288,6 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
     // ============================================================ producer (both CTAs)
     // Reads tiles from the ring and issues this CTA's loads, one stage per k-block.  The whole
     // warp runs the loop on warp-uniform values; one elected lane issues each instruction.
-#ifdef MOE_TIMING_PROBE
-    int dbg_p = 0;
-#endif
     int islot = 0;
     unsigned iph = 0;
     unsigned stage = 0, par = 1;                           // parity of "stage is free"
@@ -315,20 +313,8 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       const LoadPlan lp = make_plan(args, &args.ops[ti.slot], ti, rank);
       bool fail = false;
       for (int kb = 0; kb < ti.kblocks; ++kb) {
-#ifdef MOE_TIMING_PROBE
-        const long long p0 = clock64();
-#endif
         if (!wwait(c, &sc->empty[stage], par, 5)) { fail = true; break; }
-#ifdef MOE_TIMING_PROBE
-        const long long p1 = clock64();
-#endif
         issue_kblock(sc, stages_addr, lp, kb, stage, leader, full0_addr);
-#ifdef MOE_TIMING_PROBE
-        if (blockIdx.x == 14 + rank && lane == 0 && dbg_p < 4096) {
-          long long* pp = args.dbg + 16384 * (1 + rank) + (size_t)dbg_p++ * 4;
-          pp[0] = p0; pp[1] = p1; pp[2] = clock64(); pp[3] = ti.kind * 100000 + ti.rows * 100 + kb;
-        }
-#endif
         if (++stage == kNS) { stage = 0; par ^= 1u; }
       }
       if (fail) break;
@@ -338,11 +324,6 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
     // The whole warp runs the loops with warp-uniform values and one elected lane issues each
     // MMA and commit: per k-block one barrier wait, four MMAs and one commit, which keeps
     // issuing ahead of the tensor pipe (about 512 clocks per k-block of a 256-row tile).
-#ifdef MOE_TIMING_PROBE
-    int dbg_i = 0;
-    const unsigned long long g_start = gtime_ns();
-    const long long c_start = clock64();
-#endif
     int islot = 0;
     unsigned iph = 0, gcount = 0;
     unsigned stage = 0, par = 0;
@@ -364,13 +345,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
         bool ready = false;                           // the current stage was seen full by the look-ahead test
         const unsigned full0 = smem_u32(&sc->full[0]), empty0 = smem_u32(&sc->empty[0]);
         for (int kb = 0; kb < kblocks; ++kb) {
-#ifdef MOE_TIMING_PROBE
-          const long long q0 = clock64();
-#endif
           if (!ready && !wwait(c, &sc->full[stage], par, 8)) { fail = true; break; }
-#ifdef MOE_TIMING_PROBE
-          const long long q1 = clock64();
-#endif
           if (g1) fence_async_proxy_smem();            // this CTA's cp.async-written rows -> tensor core reads
           const unsigned sA = sbase + stage * (unsigned)kSB;
           const unsigned long long ad = umma_desc(sA, kRowBytes), bd = umma_desc(sA + kABytes, kRowBytes);
@@ -379,12 +354,6 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
           // commit that frees the stage in both CTAs, and the test of the next stage's barrier
           ready = pair_mma_kblock(d, ad, bd, idesc, kb ? 1u : 0u, empty0 + stage * 8u, full0 + nstage * 8u, npar);
           ready = __all_sync(0xffffffffu, ready) && kb + 1 < kblocks;
-#ifdef MOE_TIMING_PROBE
-          if (blockIdx.x == 14 && lane == 0 && dbg_i < 4096) {
-            long long* pp = args.dbg + (size_t)dbg_i++ * 4;
-            pp[0] = q0; pp[1] = q1; pp[2] = clock64(); pp[3] = kind * 100000 + rows * 100 + kb;
-          }
-#endif
           stage = nstage;
           par = npar;
         }
@@ -395,12 +364,6 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       if (lane == 0) mbar_arrive(&sc->iempty[islot]);
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
     }
-#ifdef MOE_TIMING_PROBE
-    if (blockIdx.x == 14 && lane == 0) {
-      args.dbg[49152] = (long long)(gtime_ns() - g_start);
-      args.dbg[49153] = clock64() - c_start;
-    }
-#endif
   } else if (warp == 1) {
     // ============================================================ gather relay (second CTA)
     // When this CTA's gather threads' copies of a stage have landed it makes them visible to the
@@ -461,11 +424,17 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       const int rpc = rows > kTileM ? 128 : 64;
       const int first = rank * rpc;                       // this CTA's first row of the tile
       int tok[kPasses];
+      const int n_rows = op->n_rows;
+      bool bad = false;
 #pragma unroll
       for (int j = 0; j < kPasses; ++j) {
         const int r = rbase + kRowsPerPass * j;
-        tok[j] = (r < rpc && first + r < rows) ? op->sorted_to_flat[row0 + first + r] / args.k : -1;
+        const int flat = (r < rpc && first + r < rows) ? op->sorted_to_flat[row0 + first + r] : 0;
+        const bool in_range = (unsigned)flat < (unsigned)n_rows;    // an index the plan never wrote is reported
+        bad |= !in_range;                                            // below and its row is skipped
+        tok[j] = (r < rpc && first + r < rows && in_range) ? flat / args.k : -1;
       }
+      if (bad) report(c.st, MOE_EBOUNDS, slot, row0, rows, 0);
       unsigned long long* landed = leader ? sc->full : sc->fullA;
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {

@@ -94,14 +94,43 @@ __device__ __noinline__ inline bool wait_counter(const Ctx& c, const int* p, int
 }
 
 // ------------------------------------------------------------------ queues
+// a slot whose plan was rejected (an expert id out of range) holds no tiles
 __device__ __forceinline__ int op_total_tiles(const OpDev* op, int fuse) {
+  if (op->plan->planned == 0) return 0;
   return op->plan->n_gemm_tiles + (fuse ? op->plan->n_comb_tiles : 0);
+}
+
+// An op without tiles (no tokens, or a plan that was rejected) never commits anything: it counts as
+// finished as soon as its own predecessor has, and its ready word is not consulted.
+__device__ inline bool op_finished(const RunArgs* a, int slot) {
+  for (int hop = 0; slot >= 0 && hop <= kMaxOps; ++hop) {
+    const OpDev* op = &a->ops[slot];
+    if (op_total_tiles(op, a->fuse_combine) > 0) return ld_acquire(&op->run->done) != 0;
+    slot = op->after_op;
+  }
+  return true;
 }
 
 __device__ inline bool op_ready(const RunArgs* a, const OpDev* op) {
   if (op->ready != nullptr && ld_acquire_sys(op->ready) == 0) return false;
-  if (op->after_op >= 0 && ld_acquire(&a->ops[op->after_op].run->done) == 0) return false;
-  return true;
+  return op_finished(a, op->after_op);
+}
+
+// Marks as done every tile-less op of the run whose chain of predecessors ends at `finished`
+// (-1: at no op at all) through tile-less ops only.  One thread; called at kernel start and when an
+// op's last tile commits.
+__device__ inline void finish_empty_ops(const RunArgs* a, int finished) {
+  for (int i = 0; i < a->n_ops; ++i) {
+    OpDev* op = &a->ops[a->slots[i]];
+    if (op_total_tiles(op, a->fuse_combine) > 0) continue;
+    int dep = op->after_op;
+    for (int hop = 0; dep >= 0 && hop <= kMaxOps && op_total_tiles(&a->ops[dep], a->fuse_combine) == 0; ++hop)
+      dep = a->ops[dep].after_op;
+    if (dep != finished) continue;
+    atomicExch(&op->run->done, 1);
+    if (op->done != nullptr) st_release_sys(op->done, 1u);
+    if (op->notify != nullptr) st_release_sys(op->notify, 1u);
+  }
 }
 
 // Claim by the whole producer warp.  1: claimed (ti filled), 0: queue exhausted, -1: the op
@@ -132,7 +161,9 @@ __device__ inline int try_claim(const RunArgs* a, QueueTables* sc, RunHead* rh, 
   t = __shfl_sync(0xffffffffu, t, 0);
   if (t >= total) return 0;
   need_ready = false;
-  if (t >= sc->cum[cls][i + 1]) {          // past the op boundary: a later op of the class
+  // the prefetched entries belong to the op at the peeked head: usable only while the ticket stays in it
+  const bool same_op = t < sc->cum[cls][i + 1];
+  if (!same_op) {                          // past the op boundary: a later op of the class
     while (t >= sc->cum[cls][i + 1]) ++i;
     slot = sc->cls_slot[cls][i];
     op = &a->ops[slot];
@@ -142,7 +173,7 @@ __device__ inline int try_claim(const RunArgs* a, QueueTables* sc, RunHead* rh, 
   // the op is instantiated by the claim of its first tile: its budget field takes effect now
   if (local == 0 && lane == 0 && op->op_budget > 0) atomicExch(&a->g->budget, op->op_budget);
   const unsigned d = t - h;
-  const bool hit = !need_ready && d < 32u;
+  const bool hit = same_op && d < 32u;
   int4 got;
   got.x = __shfl_sync(0xffffffffu, e.x, hit ? d : 0);
   got.y = __shfl_sync(0xffffffffu, e.y, hit ? d : 0);
@@ -239,6 +270,7 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
     __threadfence();
     atomicExch(&op->run->done, 1);
     if (op->done != nullptr) st_release_sys(op->done, 1u);
+    finish_empty_ops(a, ti.slot);
   }
   if (a->log_cap > 0) {
     const unsigned idx = atomicAdd(&rh->log_count, 1u);

@@ -142,26 +142,49 @@ def test_fp8_requires_scales():
     assert ei.value.code == moe.MOE_EINVAL
 
 
+def _edge_tokens(op, E):
+    """Tokens that own the first and the last row of every expert segment (tile-edge rows)."""
+    counts, offsets, s2f, _ = oracle.plan(op.ids, E)
+    k = op.ids.shape[1]
+    first = [s2f[offsets[e]] // k for e in range(E) if counts[e]]
+    last = [s2f[offsets[e + 1] - 1] // k for e in range(E) if counts[e]]
+    return np.array(first + last, dtype=np.int64)
+
+
+# share of C5's output elements that may miss the un-normalised bound 4e-2 + 4e-2 |ref| (measured: 1.8 %)
+C5_STATED_BOUND_MISS_MAX = 0.025
+
+
 def test_c5_full_size_sampled():
     """C5 in the launch configuration the bench times (4096 prefill + 512 decode tokens, one
-    persistent launch); the oracle evaluates a seeded token sample of each op.
+    persistent launch).  The oracle evaluates every decode token, the tokens that own the first and the
+    last row of every expert segment of both ops, and 256 more seeded prefill tokens.
 
-    C5's stated N(0,1) values make |y| ~ 1e5, so the 4e-2 absolute term of the acceptance
-    bound is void: an element near a zero crossing cannot be within 4 % of itself once the
-    bf16 rounding of the k expert outputs (~2e-3 of their magnitude) is added in.  The bound
-    is therefore applied to outputs normalised to unit rms: |gpu - ref| <= 4e-2 rms(ref) +
-    4e-2 |ref|, with the same relative-L2 bound of 3e-2 (measured: 2.3e-3)."""
+    C5's stated N(0,1) values make |y| ~ 1e5, so the 4e-2 absolute term of the stated bound is void: an
+    element near a zero crossing cannot be within 4 % of itself once the bf16 rounding of the k expert
+    outputs (~2e-3 of their magnitude) is added in.  Acceptance is therefore the bound applied to outputs
+    normalised to unit rms -- |gpu - ref| <= 4e-2 rms(ref) + 4e-2 |ref| -- plus the relative-L2 bound of
+    3e-2 (measured: 2.3e-3).  The share of elements that miss the bound AS STATED is computed too and held
+    below a recorded ceiling, so that it cannot grow unnoticed."""
     spec = synth.SPECS["c5"]
     W = synth.make_weights(spec, threads=16)
     ctx, bound, ops, _ = _run(spec, W=W, budget=32)
     OW = oracle_weights(spec, W)
     for b, op in zip(bound, ops):
         check_plan(b, op, spec.shape.E)
-        toks = np.random.default_rng(5).choice(op.T, size=48, replace=False).astype(np.int32)
+        if op.cls == synth.DECODE:
+            toks = np.arange(op.T, dtype=np.int32)
+        else:
+            extra = np.random.default_rng(5).choice(op.T, size=256, replace=False)
+            toks = np.unique(np.concatenate([_edge_tokens(op, spec.shape.E), extra])).astype(np.int32)
         ref = oracle.forward_tokens(OW, op.x, op.x_scale, op.ids, op.w, toks,
                                     round_A=oracle.ROUND_E4M3_1X128)
         got = b.y[torch.from_numpy(toks).long().cuda()].float().cpu().numpy()
         rms = float(np.sqrt((ref.astype(np.float64) ** 2).mean()))
         rel = assert_close(got, ref, atol=ATOL8 * max(1.0, rms), rtol=RTOL8, rel_l2=REL_L2_8)
         assert rel < 1e-2                        # far inside the bound when the quantisation is mirrored
+        err = np.abs(got.astype(np.float64) - ref.astype(np.float64))
+        miss = float((err > ATOL8 + RTOL8 * np.abs(ref)).mean())
+        print(f"c5 cls={op.cls} tokens={len(toks)} rel_l2={rel:.3e} share outside the stated bound={miss:.4f}")
+        assert miss <= C5_STATED_BOUND_MISS_MAX
         assert torch.isfinite(b.y.float()).all()

@@ -101,16 +101,66 @@ def test_bad_expert_id_is_reported_not_fatal():
     ops = synth.make_ops(spec)
     ops[0].ids[5, 1] = 99
     b = bind_ops(ctx, ops[:1], Wd)[0]
+    b.y.fill_(7.0)
     ctx.plan(0, b)
+    # the usual asynchronous sequence goes on without a host synchronisation: nothing may fault, the
+    # run and the combine leave the rejected slot alone, and the first error is the one reported
+    ctx.run([0], fuse_combine=False)
+    ctx.combine(0)
     torch.cuda.synchronize()
     code, detail = ctx.status()
-    assert code == moe.MOE_EBADID and detail[1] == 5 * 2 + 1 and detail[2] == 99
+    assert code == moe.MOE_EBADID and detail[0] == 0 and detail[1] == 5 * 2 + 1 and detail[2] == 99
     assert ctx.status()[0] == 0            # cleared; the context stays usable
+    assert torch.all(b.y == 7.0)
+    # the rejected row has no packed position, and the unclaimed tail of the permutation is marked
+    assert int(b.flat_to_sorted[5 * 2 + 1]) == -1 and int(b.sorted_to_flat[ops[0].ids.size - 1]) == -1
+    # reading the status un-planned the slot on the host side too
+    with pytest.raises(moe.MoeError) as ei:
+        ctx.run([0], fuse_combine=True)
+    assert ei.value.code == moe.MOE_ENOTPLANNED
+    with pytest.raises(moe.MoeError) as ei:
+        ctx.combine(0)
+    assert ei.value.code == moe.MOE_ENOTPLANNED
     ops = synth.make_ops(spec)
     b = bind_ops(ctx, ops[:1], Wd)[0]
     ctx.plan(0, b)
+    ctx.run([0], fuse_combine=True)
     ctx.check()
     check_plan(b, ops[0], spec.shape.E)
+    ref = oracle.forward(oracle_weights(spec, synth.make_weights(spec)), ops[0].x, None, ops[0].ids, ops[0].w)
+    assert_close(b.y.float().cpu().numpy(), ref["y"])
+
+
+def test_permutation_entries_out_of_range_are_reported_not_followed():
+    """The kernels form no address from a permutation entry outside [0, T k): a caller who overwrites the plan's
+    outputs between moe_plan and moe_run gets MOE_EBOUNDS in the status word, from the gather of the persistent
+    kernel as from the combine, and the context stays usable."""
+    spec = SMALL
+    Wd = weights_to(synth.make_weights(spec))
+    ops = synth.make_ops(spec)
+    for n_ctas in (0, 3):
+        ctx = make_ctx(spec, n_ctas=n_ctas)
+        b = bind_ops(ctx, ops[:1], Wd)[0]
+        ctx.plan(0, b)
+        torch.cuda.synchronize()
+        keep = b.sorted_to_flat.clone()
+        b.sorted_to_flat[3] = 1 << 28
+        b.sorted_to_flat[40] = -5
+        ctx.run([0], fuse_combine=False)
+        torch.cuda.synchronize()
+        assert ctx.status()[0] == moe.MOE_EBOUNDS
+        b.sorted_to_flat.copy_(keep)
+        keep = b.flat_to_sorted.clone()
+        b.flat_to_sorted[11] = 1 << 28
+        ctx.combine(0)
+        torch.cuda.synchronize()
+        code, detail = ctx.status()
+        assert code == moe.MOE_EBOUNDS and detail[0] == 11 // 2 and detail[1] == 11 % 2
+        b.flat_to_sorted.copy_(keep)
+        ctx.run([0], fuse_combine=True)
+        ctx.check()
+        ref = oracle.forward(oracle_weights(spec, synth.make_weights(spec)), ops[0].x, None, ops[0].ids, ops[0].w)
+        assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
 # ------------------------------------------------------------------ the whole path
@@ -244,7 +294,9 @@ def test_c1_as_stated():
     OW = oracle_weights(spec, W)
     for b, op in zip(bound, ops):
         ref = oracle.forward(OW, op.x, None, op.ids, op.w)
-        assert_close(b.y.float().cpu().numpy(), ref["y"], rel_l2=1e-2)
+        # ~1e-5 outputs: the rows A and D are stored in bf16 like everywhere else, but with k = 2 and an output
+        # this far below the absolute term only the norm-wise bound binds; it is kept at the common 5e-3
+        assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
 def test_one_expert_takes_everything_and_empty_op():
@@ -332,6 +384,121 @@ def test_after_op_and_done_word():
     assert np.all(log["t_commit"] >= log["t_claim"])
 
 
+@pytest.mark.parametrize("fuse", [False, True])
+@pytest.mark.parametrize("n_ctas", [0, 3], ids=["cta_pairs", "single_ctas"])
+def test_several_free_ops_of_each_class_in_one_run(fuse, n_ctas):
+    """Two prefill ops and two decode ops, none with a ready word or a predecessor, in one launch: a ticket
+    that crosses from one op of a class into the next must fetch that op's own queue entry.  Outputs start
+    from a sentinel so that a tile that never ran shows."""
+    spec = synth.Spec("four", SMALL.shape, ((synth.PREFILL, 300), (synth.DECODE, 37), (synth.PREFILL, 211),
+                                            (synth.DECODE, 5)), "softmax_topk", None, 1.0, -1.0, 22)
+    W = synth.make_weights(spec)
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec, max_tokens=300, max_ops=4, n_ctas=n_ctas, tile_log_entries=1 << 14)
+    bound = bind_ops(ctx, ops, weights_to(W))
+    for b in bound:
+        b.y.fill_(float("nan"))
+    for s, b in enumerate(bound):
+        ctx.plan(s, b)
+    ctx.set_budget(2)
+    ctx.run([0, 1, 2, 3], fuse_combine=fuse)
+    if not fuse:
+        for s in range(4):
+            ctx.combine(s)
+    ctx.check()
+    log = ctx.tile_log()
+    OW = oracle_weights(spec, W)
+    for s, (b, op) in enumerate(zip(bound, ops)):
+        n = ctx.footprint(s)[1] - (0 if fuse else -(-op.T // 16))     # unfused: no combine tiles in the launch
+        assert sorted(log["tile"][log["slot"] == s].tolist()) == list(range(n))      # every entry exactly once
+        assert_close(b.y.float().cpu().numpy(), oracle.forward(OW, op.x, None, op.ids, op.w)["y"])
+
+
+@pytest.mark.parametrize("n_ctas", [0, 3], ids=["cta_pairs", "single_ctas"])
+def test_op_without_tokens_counts_as_finished_for_its_successors(n_ctas):
+    """A layer with an empty batch is a normal case of the one-launch multi-layer form: the empty op is done
+    as soon as its own predecessor is, its done word is set, and the op chained after it runs."""
+    spec = synth.Spec("chain", SMALL.shape, ((synth.PREFILL, 120), (synth.PREFILL, 0), (synth.DECODE, 33)),
+                      "softmax_topk", None, 1.0, -1.0, 23)
+    W = synth.make_weights(spec)
+    Wd = weights_to(W)
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec, max_tokens=120, max_ops=3, n_ctas=n_ctas, wait_limit_us=200000, tile_log_entries=4096)
+    done = torch.zeros(3, dtype=torch.int32, device="cuda")
+    b0 = bind_ops(ctx, ops[0:1], Wd, done=done[0:1])[0]
+    b1 = bind_ops(ctx, ops[1:2], Wd, done=done[1:2], after_op=0)[0]
+    b2 = bind_ops(ctx, ops[2:3], Wd, done=done[2:3], after_op=1)[0]
+    for s, b in enumerate((b0, b1, b2)):
+        ctx.plan(s, b)
+    ctx.run([0, 1, 2], fuse_combine=True)
+    ctx.check()
+    assert done.tolist() == [1, 1, 1]
+    log = ctx.tile_log()
+    # the last op waited for the first one through the empty one
+    assert log["t_commit"][log["slot"] == 2].min() >= log["t_commit"][log["slot"] == 0].max()
+    OW = oracle_weights(spec, W)
+    for b, op in ((b0, ops[0]), (b2, ops[2])):
+        assert_close(b.y.float().cpu().numpy(), oracle.forward(OW, op.x, None, op.ids, op.w)["y"])
+    # an empty op with nothing before it is done at once
+    done.zero_()
+    b1f = bind_ops(ctx, ops[1:2], Wd, done=done[1:2])[0]
+    ctx.plan(1, b1f)
+    ctx.run([1, 2], fuse_combine=True)
+    ctx.check()
+    assert done.tolist() == [0, 1, 1]
+
+
+def test_ready_word_written_by_the_host_while_the_kernel_runs():
+    """Section 4.2 / 4.3: an operation becomes ready through a system-scope word.  Here the word lives in
+    pinned host memory that the device reads in place: the kernel is launched with the decode op not ready,
+    the host waits until the kernel itself reports progress (the prefill op's notify word, also in host
+    memory), then sets the ready word.  Every device wait is bounded (50 ms), so a lost write would end in
+    MOE_ETIMEOUT, not in a hang.  Outputs equal the both-ready run bit for bit."""
+    import time
+    spec = synth.Spec("hostready", synth.Shape(32, 4, 1024, 512), ((synth.PREFILL, 8192), (synth.DECODE, 64)),
+                      "zipf", 1.0, 1.0, -1.0, 47)
+    W = weights_to(synth.make_weights(spec))
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec, max_tokens=8192, max_ops=2, wait_limit_us=50000, tile_log_entries=1 << 15)
+    plain = bind_ops(ctx, ops, W)
+    for s, b in enumerate(plain):
+        ctx.plan(s, b)
+    ctx.run([0, 1], fuse_combine=True)
+    ctx.check()
+    y_ref = [b.y.clone() for b in plain]
+    n_pre = ctx.footprint(0)[1]
+    words = torch.zeros(2, dtype=torch.int32).pin_memory()        # [0] ready (host -> device), [1] notify (device -> host)
+    host = words.numpy()
+    from gpu_util import upload
+    d0, d1 = upload(ops[0], None, "cuda:0"), upload(ops[1], None, "cuda:0")
+    pre = ctx.bind(ops[0].cls, d0["x"], d0["ids"], d0["w"], W.w_gate_up, W.w_down, notify=words[1:2],
+                   notify_after=max(1, n_pre // 8))
+    dec = ctx.bind(ops[1].cls, d1["x"], d1["ids"], d1["w"], W.w_gate_up, W.w_down, ready=words[0:1])
+    ctx.plan(0, pre)
+    ctx.plan(1, dec)
+    torch.cuda.synchronize()
+    ctx.run([0, 1], fuse_combine=True)
+    t0 = time.perf_counter()
+    while host[1] == 0 and time.perf_counter() - t0 < 5.0:        # the kernel is running: it has committed tiles
+        pass
+    assert host[1] == 1
+    host[0] = 1                                                   # the host makes the decode op ready
+    ctx.check()
+    assert torch.equal(pre.y, y_ref[0]) and torch.equal(dec.y, y_ref[1])
+    log = ctx.tile_log()
+    p, d = log[log["slot"] == 0], log[log["slot"] == 1]
+    assert len(d) == ctx.footprint(1)[1]
+    # no decode tile was handed out before the kernel had told the host to go ahead
+    t_notify = np.sort(p["t_commit"])[max(1, n_pre // 8) - 1]
+    assert d["t_claim"].min() >= t_notify - 2000
+    # a ready word that the host never sets ends in a status, not a hang
+    host[:] = 0
+    ctx.run([0, 1], fuse_combine=True)
+    torch.cuda.synchronize()
+    assert ctx.status()[0] == moe.MOE_ETIMEOUT
+    assert host[1] == 1
+
+
 # ------------------------------------------------------------------ full-size configs
 
 @pytest.fixture(scope="module")
@@ -367,31 +534,59 @@ def test_c2_decode_only_full(big_weights):
     assert_close(b.y.float().cpu().numpy(), ref["y"])
 
 
-@pytest.mark.parametrize("name,fuse", [("c3", True), ("c4", True), ("c4", False)])
-def test_full_size_sampled(big_weights, name, fuse):
-    """C3 / one C4 layer in the launch configuration the bench times; the oracle evaluates
-    every decode token, the rows at every expert-segment edge and a seeded token sample."""
-    _, W, Wd = big_weights
-    spec = synth.SPECS[name]
-    ops = synth.make_ops(spec, layer=1)
-    ctx = make_ctx(spec)
-    bound = bind_ops(ctx, ops, Wd)
-    ctx.set_budget(32)
-    for s, b in enumerate(bound):
-        ctx.plan(s, b)
-    ctx.run(list(range(len(bound))), fuse_combine=fuse)
-    if not fuse:
-        for s in range(len(bound)):
-            ctx.combine(s)
-    ctx.check()
-    OW = oracle_weights(spec, W)
+def _check_sampled(ctx, spec, bound, ops, OW, n_extra=128, cap=900):
     for s, (b, op) in enumerate(zip(bound, ops)):
         counts = check_plan(b, op, spec.shape.E)
         check_tiles(ctx, s, counts)
         toks = np.arange(op.T, dtype=np.int32) if op.cls == synth.DECODE and op.T <= 256 \
-            else _sample_tokens(op, spec.shape.E, 128, 11)
-        toks = toks[:700]
+            else _sample_tokens(op, spec.shape.E, n_extra, 11)
+        toks = toks[:cap]
         ref = oracle.forward_tokens(OW, op.x, None, op.ids, op.w, toks)
         got = b.y[torch.from_numpy(toks).long().cuda()].float().cpu().numpy()
         assert_close(got, ref)
         assert torch.isfinite(b.y.float()).all()
+
+
+@pytest.mark.parametrize("fuse", [True, False])
+def test_c3_full_size_sampled(big_weights, fuse):
+    """C3 in the launch configuration the bench times; the oracle evaluates the rows at every
+    expert-segment edge and a seeded token sample."""
+    spec, W, Wd = big_weights
+    ops = synth.make_ops(spec)
+    ctx = make_ctx(spec)
+    bound = bind_ops(ctx, ops, Wd)
+    ctx.plan(0, bound[0])
+    ctx.run([0], fuse_combine=fuse)
+    if not fuse:
+        ctx.combine(0)
+    ctx.check()
+    _check_sampled(ctx, spec, bound, ops, oracle_weights(spec, W))
+
+
+def test_c4_full_size_layers_budgets_and_both_weight_sets():
+    """C4 as the bench runs it: layer 0 at decode budgets 16 and 64 (bit-identical outputs), layer 1 at
+    budget 32 on the second weight set; on each the oracle evaluates every decode token, the rows at every
+    expert-segment edge of the prefill op and a seeded token sample."""
+    spec = synth.SPECS["c4"]
+    ctx = make_ctx(spec)
+    for layer, budgets in ((0, (16, 64)), (1, (32,))):
+        W = synth.make_weights(spec, layer=layer, threads=16)
+        Wd = weights_to(W)
+        OW = oracle_weights(spec, W)
+        ops = synth.make_ops(spec, layer=layer)
+        bound = bind_ops(ctx, ops, Wd)
+        ys = []
+        for q in budgets:
+            for b in bound:
+                b.y.zero_()
+            ctx.set_budget(q)
+            for s, b in enumerate(bound):
+                ctx.plan(s, b)
+            ctx.run([0, 1], fuse_combine=True)
+            ctx.check()
+            ys.append([b.y.clone() for b in bound])
+        for other in ys[1:]:
+            assert all(torch.equal(a, b) for a, b in zip(ys[0], other))
+        _check_sampled(ctx, spec, bound, ops, OW, n_extra=96, cap=640)
+        del W, Wd, OW, bound
+        torch.cuda.empty_cache()

@@ -300,6 +300,80 @@ def test_fp8_path_equals_dense_on_dequantised_inputs():
     assert 1e-3 < rel < 6e-2
 
 
+def _deq_blocks(q, s, br, bc):
+    v = q.view(torch.float8_e4m3fn).to(torch.float64)
+    return v * s.to(torch.float64).repeat_interleave(br, -2).repeat_interleave(bc, -1)
+
+
+def _quant_rows_torch(A: torch.Tensor, group: int) -> torch.Tensor:
+    """Library restatement of the on-path quantisation: per row and per `group` consecutive columns one
+    fp32 scale amax/448 (1 for an all-zero group), codes by torch's float8_e4m3fn cast of v * (448/amax),
+    returned dequantised (code * scale) in float64."""
+    n, I = A.shape
+    blk = A.to(torch.float32).view(n, I // group, group)
+    amax = blk.abs().amax(dim=2, keepdim=True)
+    scale = torch.where(amax > 0, amax / np.float32(448.0), torch.ones_like(amax))
+    inv = torch.where(amax > 0, np.float32(448.0) / amax, torch.zeros_like(amax))
+    codes = (blk * inv).clamp(-448.0, 448.0).to(torch.float8_e4m3fn)
+    return (codes.to(torch.float32) * scale).view(n, I).to(torch.float64)
+
+
+@pytest.mark.parametrize("I", [256, 384])
+def test_mirrored_e4m3_rounding_of_the_intermediate_is_per_row_per_128_columns(I):
+    """The one quantisation on the FP8 path: the SwiGLU output goes to e4m3 with one fp32 scale per row and
+    per 128 consecutive columns (scale = amax/448) BEFORE the down projection.  With two or three groups per
+    row, the oracle's rounded result must equal: its own un-rounded intermediate, quantised here with torch's
+    e4m3 cast, times the dequantised down weights in float64.  A wrong group width, a wrong scale constant or a
+    quantisation placed elsewhere on the path breaks the equality; the negative controls show the test sees them."""
+    spec = synth.scaled(synth.SPECS["c5"], shape=synth.Shape(3, 2, 256, I, "fp8"), ops=((synth.PREFILL, 7),))
+    sh = spec.shape
+    Wt = synth.make_weights(spec, threads=2)
+    op = synth.make_ops(spec)[0]
+    W = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wt.w_gate_up, Wt.w_down, Wt.s_gate_up, Wt.s_down)
+    row_token = np.repeat(np.arange(op.T, dtype=np.int32), sh.k)
+    row_expert = op.ids.reshape(-1)
+    _, A = oracle.ffn_rows(W, op.x, op.x_scale, row_token, row_expert, want_A=True)
+    D_q = oracle.ffn_rows(W, op.x, op.x_scale, row_token, row_expert, round_A=oracle.ROUND_E4M3_1X128)
+    w2 = _deq_blocks(Wt.w_down, Wt.s_down, 128, 128)               # [E, H, I] float64
+
+    def down(Aq):
+        return np.stack([(w2[int(e)] @ Aq[r]).numpy() for r, e in enumerate(row_expert)])
+
+    scale = np.abs(D_q).max()
+    expect = down(_quant_rows_torch(torch.from_numpy(A), 128))
+    assert np.abs(D_q - expect).max() <= 1e-6 * scale
+    # negative controls: one group per row, 64-wide groups, a scale of amax/240, and no rounding at all
+    assert np.abs(D_q - down(_quant_rows_torch(torch.from_numpy(A), I))).max() > 1e-3 * scale
+    assert np.abs(D_q - down(_quant_rows_torch(torch.from_numpy(A), 64))).max() > 1e-3 * scale
+    assert np.abs(D_q - down(torch.from_numpy(A).to(torch.float64))).max() > 1e-3 * scale
+    blk = torch.from_numpy(A).view(A.shape[0], I // 128, 128)
+    amax = blk.abs().amax(dim=2, keepdim=True)
+    wrong = ((blk * (240.0 / amax)).to(torch.float8_e4m3fn).to(torch.float32) * (amax / 240.0)).view(A.shape)
+    assert np.abs(D_q - down(wrong.to(torch.float64))).max() > 1e-3 * scale
+
+
+def test_bf16_rounding_switches_match_the_library_cast():
+    """round_A / round_D = bf16 (the switches that localise a GPU mismatch to the stored intermediate or the
+    stored expert output): A is cast to bf16 before the down projection, D after it -- each against torch's
+    bfloat16 cast applied to the oracle's un-rounded values, the down projection redone in float64."""
+    spec = synth.Spec("rb", synth.Shape(3, 2, 256, 384), ((synth.PREFILL, 6),), "uniform", None, 1.0, -1.0, 91)
+    sh = spec.shape
+    Wt = synth.make_weights(spec, threads=2)
+    op = synth.make_ops(spec)[0]
+    W = oracle.Weights(sh.E, sh.k, sh.H, sh.I, Wt.w_gate_up, Wt.w_down)
+    row_token = np.repeat(np.arange(op.T, dtype=np.int32), sh.k)
+    row_expert = op.ids.reshape(-1)
+    D, A = oracle.ffn_rows(W, op.x, None, row_token, row_expert, want_A=True)
+    w2 = Wt.w_down.to(torch.float64)
+    A_b = torch.from_numpy(A).to(torch.bfloat16).to(torch.float64)
+    expect_A = np.stack([(w2[int(e)] @ A_b[r]).numpy() for r, e in enumerate(row_expert)])
+    got_A = oracle.ffn_rows(W, op.x, None, row_token, row_expert, round_A=oracle.ROUND_BF16)
+    assert np.abs(got_A - expect_A).max() <= 1e-6 * np.abs(expect_A).max()
+    assert np.abs(got_A - D).max() > 1e-4 * np.abs(D).max()         # the rounding is visible
+    got_D = oracle.ffn_rows(W, op.x, None, row_token, row_expert, round_D=oracle.ROUND_BF16)
+    assert np.array_equal(got_D, torch.from_numpy(D).to(torch.bfloat16).float().numpy())
+
+
 def test_online_budget_closed_forms_and_brute_force():
     """Section 6.4: q' = min(Q_max, ceil_c(q x_moe / x_moe*)).  Closed forms, and exact rational arithmetic
     on a grid (a wrong rounding direction, a forgotten cap or a forgotten cluster multiple fails one)."""
