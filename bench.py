@@ -134,6 +134,7 @@ class Workload:
     """Device-resident inputs of one workload plus the calls of one step."""
 
     def __init__(self, name: str, rank: int, device: torch.device, tile_log: int = 0):
+        """Generates the workload's seeded inputs on the host, uploads them and plans nothing yet."""
         import paper_2607_18002_b200 as moe
         self.moe = moe
         self.name = name
@@ -227,6 +228,28 @@ class Workload:
             self.layers2.append((ops, b2, host))
         self.s_h2d, self.s_comp, self.s_d2h = (torch.cuda.Stream(device=device) for _ in range(3))
 
+    def run_e2e_serial(self, steps: int):
+        """The same end-to-end step on ONE stream, nothing overlapped: copy in, plan, run, copy out, and the
+        host waits for the result before it starts the next step.  The difference to run_e2e is what the
+        copies cost when they are not hidden behind the neighbouring steps' kernels."""
+        ctx = self.ctx
+        for _ in range(steps):
+            for li, (_, bound, host) in enumerate(self.layers):
+                for b, (hx, hi, hw, hy, hs) in zip(bound, host):
+                    b.x.copy_(hx, non_blocking=True)
+                    if hs is not None:
+                        b.x_scale.copy_(hs, non_blocking=True)
+                    b.topk_ids.copy_(hi, non_blocking=True)
+                    b.topk_w.copy_(hw, non_blocking=True)
+                if self.spec.layers > 1:
+                    ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
+                for s_, b in enumerate(bound):
+                    ctx.plan(s_, b)
+                ctx.run(list(range(len(bound))), fuse_combine=True)
+                for b, (_, _, _, hy, _) in zip(bound, host):
+                    hy.copy_(b.y, non_blocking=True)
+            torch.cuda.synchronize(self.device)
+
     def run_e2e(self, steps: int):
         """`steps` steps with host buffers: every step copies its inputs from pinned host memory,
         plans, runs and copies its result back to pinned host memory.  Copies and kernels run on
@@ -298,8 +321,15 @@ def oracle_sample(w: Workload, seconds_target: float = 12.0):
                            f"seeded tokens of {w.name} ({last_dt:.2f} s)")
 
 
+def _pcts(v):
+    return {"n": int(len(v)), "p50_us": float(np.percentile(v, 50)), "p99_us": float(np.percentile(v, 99)),
+            "mean_us": float(v.mean()), "max_us": float(v.max())}
+
+
 def _log_summary(log):
-    """Service time (claim -> commit) per class and tile kind, CTA occupancy and idle gaps."""
+    """Per class and tile kind, two readings of a tile's time from the kernel's tile log: its SERVICE time
+    (claim -> commit) and its LATENCY (the moment it could first have run -> commit; every op of these
+    launches is ready at launch, so that moment is the launch's first claim).  Plus op spans, CTA occupancy."""
     out = {"records": int(len(log))}
     if len(log) == 0:
         return out
@@ -307,6 +337,7 @@ def _log_summary(log):
     span = (int(log["t_commit"].max()) - t0) / 1e3
     out["kernel_span_us"] = span
     service = (log["t_commit"].astype(np.int64) - log["t_claim"].astype(np.int64)) / 1e3
+    latency = (log["t_commit"].astype(np.int64) - t0) / 1e3
     names = {0: "gate_up", 1: "down", 2: "combine"}
     for cls, cname in ((0, "decode"), (1, "prefill")):
         mc = log["cls"] == cls
@@ -314,17 +345,14 @@ def _log_summary(log):
             continue
         gemm = mc & (log["kind"] < 2)
         if gemm.any():
-            v = service[gemm]
-            out[f"{cname}_tile"] = {"n": int(gemm.sum()), "p50_us": float(np.percentile(v, 50)),
-                                    "p99_us": float(np.percentile(v, 99)), "max_us": float(v.max())}
-        out[f"{cname}_op_us"] = float((int(log["t_commit"][mc].max()) - int(log["t_claim"][mc].min())) / 1e3)
+            out[f"{cname}_tile"] = _pcts(service[gemm])
+            out[f"{cname}_tile_latency"] = _pcts(latency[gemm])
+        out[f"{cname}_op_us"] = float((int(log["t_commit"][mc].max()) - t0) / 1e3)
         out[f"{cname}_first_claim_us"] = float((int(log["t_claim"][mc].min()) - t0) / 1e3)
         for kind, kname in names.items():
             m = mc & (log["kind"] == kind)
             if m.any():
-                v = service[m]
-                out[f"{cname}_{kname}"] = {"n": int(m.sum()), "p50_us": float(np.percentile(v, 50)),
-                                           "p99_us": float(np.percentile(v, 99)), "mean_us": float(v.mean())}
+                out[f"{cname}_{kname}"] = _pcts(service[m])
     ctas = np.unique(log["cta"])
     out["ctas_with_tiles"] = int(len(ctas))
     # busy time per CTA = union of its (overlapping) tile intervals
@@ -342,26 +370,75 @@ def _log_summary(log):
     return out
 
 
+def _ratios(co, iso):
+    """Co-run over isolated, for both readings of a decode tile's time and for the whole decode op."""
+    r = {}
+    if "decode_tile" in co and "decode_tile" in iso:
+        for key, name in (("decode_tile", "service"), ("decode_tile_latency", "latency")):
+            r[f"decode_tile_{name}_p50_ratio"] = co[key]["p50_us"] / iso[key]["p50_us"]
+            r[f"decode_tile_{name}_p99_ratio"] = co[key]["p99_us"] / iso[key]["p99_us"]
+        r["decode_op_ratio"] = co["decode_op_us"] / iso["decode_op_us"]
+        r["decode_op_us"] = {"corun": co["decode_op_us"], "isolated": iso["decode_op_us"]}
+        if "prefill_op_us" in co:
+            r["prefill_op_us_corun"] = co["prefill_op_us"]
+    return r
+
+
 def tile_stats(w: Workload):
-    """Per-tile timing of one extra (untimed) step from the kernel's tile log: the analogue of
-    the paper's preemption-interval measurement; for a co-scheduled workload also the decode
-    tiles alone (same budget, no prefill op in the launch) for the co-run / isolated ratio."""
-    w.step()
-    w.ctx.check()
-    log = w.ctx.tile_log()
-    out = {"corun": _log_summary(log)}
-    _, bound, _ = w.layers[-1]
+    """Per-tile timing from the kernel's tile log (extra, untimed launches): the analogue of the paper's
+    preemption-interval measurement (Section 7.6).  For a co-scheduled workload, one layer per decode budget
+    of the workload is launched twice -- both ops together, then the decode op alone at the same budget
+    ("isolated") -- and the decode tiles' times are compared under both readings (service: claim -> commit;
+    latency: launch -> commit), next to the decode op's completion time."""
+    ctx = w.ctx
+    mixed = any(len(bound) > 1 for _, bound, _ in w.layers)
+    if not mixed:
+        w.step()
+        ctx.check()
+        return {"corun": _log_summary(ctx.tile_log())}
+    out = {"per_budget": {}}
+    budgets = synth.C4_BUDGETS if w.spec.layers > 1 else (None,)
+    pooled = {"co": [], "iso": []}
+    for li, q in enumerate(budgets):
+        if li >= len(w.layers):
+            break
+        _, bound, _ = w.layers[li]
+        dec = [s for s, b in enumerate(bound) if b.c.cls == 0]
+        if q is not None:
+            ctx.set_budget(q)
+        for s, b in enumerate(bound):
+            ctx.plan(s, b)
+        ctx.run(list(range(len(bound))), fuse_combine=True)
+        ctx.check()
+        log_co = ctx.tile_log()
+        co = _log_summary(log_co)
+        ctx.run(dec, fuse_combine=True)
+        ctx.check()
+        log_iso = ctx.tile_log()
+        iso = _log_summary(log_iso)
+        entry = {"layer": li, "corun": co, "decode_isolated": iso}
+        entry.update(_ratios(co, iso))
+        out["per_budget"][str(q)] = entry
+        for key, lg in (("co", log_co), ("iso", log_iso)):
+            m = (lg["cls"] == 0) & (lg["kind"] < 2)
+            t0 = int(lg["t_claim"].min())
+            pooled[key].append(np.stack([(lg["t_commit"][m].astype(np.int64) - lg["t_claim"][m].astype(np.int64)) / 1e3,
+                                         (lg["t_commit"][m].astype(np.int64) - t0) / 1e3]))
+    co, iso = np.concatenate(pooled["co"], axis=1), np.concatenate(pooled["iso"], axis=1)
+    for i, name in enumerate(("service", "latency")):
+        out[f"decode_tile_{name}_p50_ratio"] = float(np.percentile(co[i], 50) / np.percentile(iso[i], 50))
+        out[f"decode_tile_{name}_p99_ratio"] = float(np.percentile(co[i], 99) / np.percentile(iso[i], 99))
+        out[f"decode_tile_{name}_us"] = {"corun_p50": float(np.percentile(co[i], 50)), "corun_p99": float(np.percentile(co[i], 99)),
+                                         "isolated_p50": float(np.percentile(iso[i], 50)),
+                                         "isolated_p99": float(np.percentile(iso[i], 99))}
+    out["decode_op_ratio"] = {q: e["decode_op_ratio"] for q, e in out["per_budget"].items() if "decode_op_ratio" in e}
+    out["readings"] = ("service = commit - claim of a decode tile; latency = commit - launch start (all ops ready at "
+                       "launch); isolated = the same decode op alone in the launch at the same budget")
+    _, bound, _ = w.layers[min(1, len(w.layers) - 1)]
     dec = [s for s, b in enumerate(bound) if b.c.cls == 0]
-    if dec and len(dec) < len(bound):
-        w.ctx.run(dec, fuse_combine=True)
-        w.ctx.check()
-        iso = _log_summary(w.ctx.tile_log())
-        out["decode_isolated"] = iso
-        if "decode_tile" in iso and "decode_tile" in out["corun"]:
-            out["decode_tile_p99_ratio"] = out["corun"]["decode_tile"]["p99_us"] / iso["decode_tile"]["p99_us"]
-            out["decode_tile_p50_ratio"] = out["corun"]["decode_tile"]["p50_us"] / iso["decode_tile"]["p50_us"]
-            out["decode_op_ratio"] = out["corun"]["decode_op_us"] / iso["decode_op_us"]
-        out["decode_arrives_mid_prefill"] = _mid_run_arrival(w, bound, dec)
+    if w.spec.layers > 1:
+        ctx.set_budget(synth.C4_BUDGETS[1])
+    out["decode_arrives_mid_prefill"] = _mid_run_arrival(w, bound, dec)
     return out
 
 
@@ -374,6 +451,7 @@ def _mid_run_arrival(w: Workload, bound, dec):
     pre = [s for s in range(len(bound)) if s not in dec]
     ps, ds = pre[0], dec[0]
     word = torch.zeros(1, dtype=torch.int32, device=w.device)
+    w.ctx.plan(ps, bound[ps])
     n_pre = w.ctx.footprint(ps)[1]
     after = max(1, n_pre // 3)
     bp, bd = bound[ps], bound[ds]
@@ -493,17 +571,17 @@ def run_reference(args):
         "gpu_launches": 0}))
 
 
-def run_ours(args):
-    from paper_2607_18002_b200 import dist
-    if not torch.cuda.is_available():
-        raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
-    rank, world, local = dist.init_from_env()
-    device = torch.device("cuda", local)
-    torch.cuda.set_device(device)
-    peaks, peak_src = load_peaks()
-    w = Workload(args.workload, rank, device, tile_log=(1 << 17) if args.tile_log else 0)
-    K, Wm = args.steps, args.warmup
+# steps / warm-up of the workloads that ride along with the default run (one JSON line for all targets)
+SUB_STEPS = {"c2": (100, 5), "c4": (2, 3), "c5": (15, 4)}
 
+
+def measure(name: str, args, K: int, Wm: int, rank: int, world: int, local: int, device, peaks, peak_src,
+            tile_log: bool, e2e: bool, one_launch: bool):
+    """Times one workload: device-resident steps (CUDA events, barrier on both sides), the live duration of
+    every persistent launch for the roofline, optionally the end-to-end loops with host buffers and the
+    tile-log statistics.  Returns the fields of a bench line."""
+    from paper_2607_18002_b200 import dist
+    w = Workload(name, rank, device, tile_log=(1 << 17) if tile_log else 0)
     for _ in range(Wm):
         w.step()
     w.ctx.check()
@@ -527,19 +605,33 @@ def run_ours(args):
     ms_per_step = 1e3 * dist.reduce_scalar(secs, "max") / K
 
     # ---- end to end with host buffers (host clock around K steps, everything synchronised on both sides)
-    w.run_e2e(min(Wm, 3))
-    dist.barrier()
-    torch.cuda.synchronize()
-    t_e2e = time.perf_counter()
-    w.run_e2e(K)
-    t_e2e = time.perf_counter() - t_e2e
-    dist.barrier()
-    w.ctx.check()
-    w.ctx2.check()
-    e2e_value = dist.job_throughput(w.flops * K, t_e2e) / 1e12
+    e2e_out = e2e_serial = None
+    if e2e:
+        w.run_e2e(min(Wm, 3))
+        dist.barrier()
+        torch.cuda.synchronize()
+        t_e2e = time.perf_counter()
+        w.run_e2e(K)
+        t_e2e = time.perf_counter() - t_e2e
+        dist.barrier()
+        w.ctx.check()
+        w.ctx2.check()
+        e2e_out = {"value": dist.job_throughput(w.flops * K, t_e2e) / 1e12, "unit": UNIT,
+                   "h2d_bytes_per_step": w.h2d, "d2h_bytes_per_step": w.d2h,
+                   "how": "two buffer sets over three streams: a step's copies overlap the neighbouring steps' kernels"}
+        Ks = max(3, K // 3)
+        w.run_e2e_serial(2)
+        dist.barrier()
+        t_ser = time.perf_counter()
+        w.run_e2e_serial(Ks)
+        t_ser = time.perf_counter() - t_ser
+        dist.barrier()
+        w.ctx.check()
+        e2e_serial = {"value": dist.job_throughput(w.flops * Ks, t_ser) / 1e12, "unit": UNIT, "steps": Ks,
+                      "ms_per_step": 1e3 * t_ser / Ks,
+                      "how": "one stream, nothing overlapped, the host waits for every step's result"}
 
     # ---- roofline of the dominant kernel (the persistent kernel), from live CUDA events
-    launches = len(run_ms)
     t_run = float(np.mean(run_ms)) / 1e3
     kernel_name = "moe_apk_pair_kernel" if w.ctx.ctas_per_tile == 2 else "moe_apk_kernel"
     flops_launch = w.flops / len(w.layers)
@@ -551,16 +643,16 @@ def run_ours(args):
     tpeak = peaks["bf16_tflops_sustained" if long_step else "bf16_tflops"] * (2.0 if w.fp8 else 1.0)
     tensor_frac = flops_launch / t_run / 1e12 / tpeak
     hbm_frac = bytes_launch / t_run / 1e9 / peaks["hbm_gbs"]
-    if args.workload in ("c2", "c2s", "c5", "c5s"):
+    if name in ("c2", "c2s", "c5", "c5s"):
         roof = {"bound": "hbm", "achieved": bytes_launch / t_run / 1e9, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": hbm_frac}
     else:
         roof = {"bound": "tensor", "achieved": flops_launch / t_run / 1e12,
                 "peak": tpeak, "unit": "TFLOP/s", "frac": tensor_frac}
-    roof.update({"traffic": NCU_DRAM_BYTES.get((args.workload, kernel_name)), "kernel": kernel_name,
+    roof.update({"traffic": NCU_DRAM_BYTES.get((name, kernel_name)), "kernel": kernel_name,
                  "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of the small variant, "
                                    "scaled by active experts (see profiles/)"
-                                   if (args.workload, kernel_name) in NCU_DRAM_BYTES else None,
+                                   if (name, kernel_name) in NCU_DRAM_BYTES else None,
                  "peak_source": peak_src, "peak_kind": "sustained" if long_step else "burst",
                  "launch_ms_mean": 1e3 * t_run, "launch_ms_min": float(np.min(run_ms)),
                  "algorithmic_flops_per_launch": flops_launch,
@@ -569,31 +661,68 @@ def run_ours(args):
                  "tensor_frac_of_sustained": flops_launch / t_run / 1e12 / (peaks["bf16_tflops_sustained"] * (2.0 if w.fp8 else 1.0)),
                  "hbm_frac": hbm_frac})
 
-    tiles = tile_stats(w) if args.tile_log else None
-    one_launch = persistent_layers(w, K, Wm) if (args.one_launch and len(w.layers) > 1 and world == 1) else None
+    tiles = tile_stats(w) if tile_log else None
+    one = persistent_layers(w, K, Wm) if (one_launch and len(w.layers) > 1 and world == 1) else None
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and e2e:
         v, cores, sample = oracle_sample(w)
         cpu = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample}
 
+    sh = w.sh
+    res = {"value": value, "unit": UNIT, "steps": K, "warmup": Wm, "ms_per_step": ms_per_step,
+           "dtype": "fp8_e4m3" if w.fp8 else "bf16",
+           "config": {"workload": name, "ops": [[c, t] for c, t in w.spec.ops],
+                      "layers": w.spec.layers, "experts": sh.E, "top_k": sh.k, "hidden": sh.H,
+                      "inter": sh.I, "l2": "inputs_exceed_l2 (weights >> 126 MB, no flush)",
+                      "buffers": "the same X / y buffers every step: the step's 7-10 GB of weights pass through "
+                                 "the 126 MB L2 between two uses of a buffer",
+                      "replicas": world, "fused_combine": True},
+           "clocks": clk.summary(), "gpu_launches": w.launches_per_step * K, "roofline": roof}
+    if e2e_out:
+        res["e2e"], res["e2e_serial"] = e2e_out, e2e_serial
+    if cpu:
+        res["cpu_baseline"] = cpu
+    if tiles:
+        res["tiles"] = tiles
+    if one:
+        res["one_launch_for_all_layers"] = one
+    del w
+    torch.cuda.empty_cache()
+    return res
+
+
+def run_ours(args):
+    from paper_2607_18002_b200 import dist
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (the library has no CPU path)")
+    rank, world, local = dist.init_from_env()
+    device = torch.device("cuda", local)
+    torch.cuda.set_device(device)
+    peaks, peak_src = load_peaks()
+    main_res = measure(args.workload, args, args.steps, args.warmup, rank, world, local, device, peaks, peak_src,
+                       tile_log=args.tile_log, e2e=True, one_launch=args.one_launch)
+    # The default run also measures the other targets of the metric on their own workloads: the decode-only
+    # layer (HBM), the mixed 8-layer stream (decode-tile latency under prefill, from the tile log) and the
+    # FP8 layer.  Each gets its own warm-up, timed region, clock record and status check.
+    sub = {}
+    if args.sub_results and world == 1:
+        for name in ("c2", "c4", "c5"):
+            if name == args.workload:
+                continue
+            k_, w_ = SUB_STEPS[name]
+            sub[name] = measure(name, args, k_, w_, rank, world, local, device, peaks, peak_src,
+                                tile_log=(name == "c4"), e2e=False, one_launch=False)
     if rank == 0:
-        sh = w.sh
-        print(json.dumps({
-            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
-            "warmup": Wm, "ms_per_step": ms_per_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "fp8_e4m3" if w.fp8 else "bf16",
-            "data": "synthetic",
-            "config": {"workload": args.workload, "ops": [[c, t] for c, t in w.spec.ops],
-                       "layers": w.spec.layers, "experts": sh.E, "top_k": sh.k, "hidden": sh.H,
-                       "inter": sh.I, "l2": "inputs_exceed_l2 (weights >> 126 MB, no flush)",
-                       "replicas": world, "fused_combine": True},
-            "clocks": clk.summary(),
-            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": w.h2d,
-                    "d2h_bytes_per_step": w.d2h},
-            "gpu_launches": w.launches_per_step * K,
-            "roofline": roof, "cpu_baseline": cpu, **({"tiles": tiles} if tiles else {}),
-            **({"one_launch_for_all_layers": one_launch} if one_launch else {})}))
+        line = {"metric": METRIC, "value": main_res.pop("value"), "unit": UNIT, "n_gpus": world,
+                "steps": main_res.pop("steps"), "warmup": main_res.pop("warmup"),
+                "ms_per_step": main_res.pop("ms_per_step"), "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": main_res.pop("dtype"), "data": "synthetic"}
+        line.update(main_res)
+        line.setdefault("cpu_baseline", None)
+        if sub:
+            line["sub_results"] = sub
+        print(json.dumps(line))
     dist.shutdown()
 
 
@@ -608,7 +737,10 @@ def main():
     ap.add_argument("--tile-log", action="store_true", help="add per-tile timing statistics of one extra untimed step")
     ap.add_argument("--one-launch", action="store_true",
                     help="multi-layer workloads: also time all layers as one persistent launch per step")
+    ap.add_argument("--no-sub", action="store_true",
+                    help="default workload only: skip the c2 / c4 / c5 sub-results")
     args = ap.parse_args()
+    args.sub_results = args.workload == "c3" and not args.no_sub
     ds, dw = DEFAULT_STEPS[args.workload]
     if args.impl == "reference":
         ds, dw = 3, 1

@@ -150,6 +150,15 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
  * bounded by wait_limit_us. */
 int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, void* stream);
 
+/* The same tiles as plain (non-persistent) launches, for measuring what the tile scheduler costs
+ * (the scheduling-overhead experiment of Section 7.4): one launch for the gate/up tiles of the op in
+ * `slot` and one for its down tiles, each with one claiming unit per queue entry -- no queue, no
+ * budget, no ready word -- then the stand-alone combine.  Same tile code, bit-identical y.  bf16 on
+ * an even grid only (MOE_EINVAL otherwise, and for an op with a ready word or a predecessor).  The
+ * grid size is the op's entry count, which lives on the device: this call SYNCHRONISES the stream to
+ * read it, so it is a measuring tool, not a serving path. */
+int moe_run_plain(moe_ctx_t* ctx, int slot, void* stream);
+
 /* Post-processing: y[t,:] = sum_j w[t,j] * D[flat_to_sorted[t*k+j],:], slots added in
  * order j = 0..k-1 in fp32 (the last step of the MoE module of Section 2.1).  A permutation
  * entry outside [0, T*k) is reported as MOE_EBOUNDS and contributes nothing. */

@@ -323,11 +323,51 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
   a.dtype = c.dtype;
   a.kb_elems = c.dtype == MOE_DTYPE_FP8_E4M3 ? 128 : kBlockK;
   a.wait_ns = (long long)c.wait_limit_us * 1000;
+  a.static_kind = -1;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
   const cudaError_t le = ctx->pair_kernel ? launch_pair(a, ctx->rh(), ctx->n_ctas, st)
                                           : launch_run(a, ctx->rh(), ctx->n_ctas, st);
   if (le != cudaSuccess) return MOE_ECUDA;
+  return MOE_OK;
+}
+
+int moe_run_plain(moe_ctx_t* ctx, int slot, void* stream) {
+  if (!ctx || slot < 0 || slot >= ctx->cfg.max_ops) return MOE_EINVAL;
+  if (!ctx->pair_kernel) return MOE_EINVAL;
+  if (!ctx->planned[slot]) return MOE_ENOTPLANNED;
+  if (ctx->ops[slot].after_op >= 0 || ctx->ops[slot].ready) return MOE_EINVAL;
+  const moe_config_t& c = ctx->cfg;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the grid is the op's entry count, which only the device knows: wait for the plan and read it
+  PlanState ps;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return MOE_ECUDA;
+  if (cudaMemcpy(&ps, ctx->slot_base(slot) + ctx->L.plan_off, sizeof(ps), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return MOE_ECUDA;
+  if (!ps.planned) return MOE_ENOTPLANNED;
+  RunArgs a;
+  memset(&a, 0, sizeof(a));
+  a.slots[0] = slot;
+  a.g = ctx->g();
+  a.ops = ctx->op_dev(0);
+  a.log = reinterpret_cast<moe_tile_rec_t*>(ctx->ws + ctx->L.log_off);
+  a.log_cap = c.tile_log_entries;
+  a.n_ops = 1;
+  a.fuse_combine = 0;
+  a.E = c.n_experts; a.k = c.top_k; a.H = c.hidden; a.I = c.inter;
+  a.dtype = c.dtype;
+  a.kb_elems = kBlockK;
+  a.wait_ns = (long long)c.wait_limit_us * 1000;
+  if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
+  if (ps.n_gemm_tiles > 0) {
+    // the down launch starts when the gate/up launch has ended (stream order), so the per-tile dependency
+    // counters it checks are already complete
+    a.static_kind = kGateUp;
+    if (launch_pair(a, ctx->rh(), 2 * ps.n_gemm_tiles, st) != cudaSuccess) return MOE_ECUDA;
+    a.static_kind = kDown;
+    if (launch_pair(a, ctx->rh(), 2 * ps.n_gemm_tiles, st) != cudaSuccess) return MOE_ECUDA;
+  }
+  if (launch_combine(ctx->op_dev(slot), ctx->ops[slot].n_tokens, c.top_k, c.hidden, st) != cudaSuccess) return MOE_ECUDA;
   return MOE_OK;
 }
 

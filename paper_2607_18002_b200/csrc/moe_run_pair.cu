@@ -261,7 +261,9 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
     ti.kind = kEnd;
     ti.slot = ti.tile = ti.m = ti.row0 = ti.rows = ti.n = ti.kblocks = ti.expert = ti.cls = 0;
     ti.t_claim = 0;
-    claim_next(c, &sc->qt, rh, lane, ti, need_ready);
+    const bool plain = args.static_kind >= 0;             // plain launch: this pair runs one given entry
+    if (plain) claim_static(&args, (int)(blockIdx.x >> 1), ti);
+    else claim_next(c, &sc->qt, rh, lane, ti, need_ready);
     while (true) {
       ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);
       const OpDev* op = &args.ops[ti.kind == kEnd ? args.slots[0] : ti.slot];
@@ -282,7 +284,8 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       if (ti.kind == kEnd || !ok) break;
       if (!wwait(c, &sc->taken[islot], iph, 26)) break;
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
-      claim_next(c, &sc->qt, rh, lane, ti, need_ready);
+      if (plain) ti.kind = kEnd;
+      else claim_next(c, &sc->qt, rh, lane, ti, need_ready);
     }
   } else if (warp == 3) {
     // ============================================================ producer (both CTAs)
@@ -586,6 +589,7 @@ cudaError_t prepare_pair_kernel() {
                               (int)pairk::kSmemBytes);
 }
 
+// n_ctas: the persistent grid, or 2 x the number of queue entries for a plain launch
 cudaError_t launch_pair(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream) {
   pairk::moe_apk_pair_kernel<<<n_ctas, pairk::kThreads, pairk::kSmemBytes, stream>>>(args, rh);
   return cudaGetLastError();

@@ -232,6 +232,28 @@ __device__ inline bool wait_op_ready(const Ctx& c, int lane, const TileInfo& ti)
   return true;
 }
 
+// The plain (non-persistent) launch: unit `unit` of the grid takes queue entry `unit` of the run's only op,
+// if that entry is of the launch's kind, and nothing else.  No queue head, no budget, no ready word.
+__device__ inline void claim_static(const RunArgs* a, int unit, TileInfo& ti) {
+  const int slot = a->slots[0];
+  const OpDev* op = &a->ops[slot];
+  ti.kind = kEnd;
+  if (unit >= op->plan->n_gemm_tiles) return;
+  const int4 got = op->tile_list[unit];
+  if (entry_kind(got) != a->static_kind) return;
+  ti.kind = entry_kind(got);
+  ti.n = entry_n(got);
+  ti.m = entry_m(got);
+  ti.row0 = got.y;
+  ti.rows = got.z;
+  ti.expert = got.w;
+  ti.slot = slot;
+  ti.tile = unit;
+  ti.cls = op->cls;
+  ti.kblocks = (ti.kind == kGateUp ? a->H : a->I) / a->kb_elems;
+  ti.t_claim = gtime_ns();
+}
+
 // Blocking form: waits (bounded) while an op exists that is not ready.  Returns with
 // ti.kind == kEnd when nothing is left (or the run was aborted).
 __device__ inline void claim_next(const Ctx& c, QueueTables* sc, RunHead* rh, int lane, TileInfo& ti,

@@ -13,6 +13,11 @@ Times are microseconds from the common start: CUDA events for separate launches;
 launch the decode operation's completion comes from the kernel's tile log.
 
     python -m paper_2607_18002_b200.sharing_study          # prints the table (needs a GPU)
+
+`scheduler_overhead` is the companion experiment of Section 7.4: the persistent kernel against plain
+launches of the same tile code, on a prefill-sized op and on decode-sized ops over 8..256 active experts.
+
+    python -m paper_2607_18002_b200.sharing_study --overhead
 """
 from __future__ import annotations
 
@@ -124,7 +129,75 @@ def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, b
     return rows
 
 
+def scheduler_overhead(E=256, k=8, H=3072, I=1536, prefill_tokens=8192, zipf_s=1.2, decode_tokens=128,
+                       actives=(8, 32, 128, 256), reps=10, seed=3, device="cuda:0"):
+    """What the persistent kernel's tile scheduling costs against plain launches of the SAME tile code
+    (the experiment of Section 7.4): for a prefill-sized op (contiguous layout, Zipf routing) and for a
+    decode-sized op over a growing number of active experts, the time of moe_run + moe_combine next to the
+    time of moe_run_plain (one gate/up launch and one down launch with a claiming unit per tile, then the
+    combine).  CUDA events, median of `reps` after one warm-up, L2 flushed between launches.  Returns rows of
+    dict(case, x_moe, persistent_us, plain_us)."""
+    import torch
+
+    import paper_2607_18002_b200 as moe
+    from workloads import synth
+
+    dev = torch.device(device)
+    spec = synth.Spec("overhead", synth.Shape(E, k, H, I), ((synth.PREFILL, prefill_tokens),), "zipf", zipf_s, 1.0, 0.02, seed)
+    W = synth.make_weights(spec)
+    w1, w2 = W.w_gate_up.to(dev), W.w_down.to(dev)
+    ctx = moe.Context(E, k, H, I, max(prefill_tokens, decode_tokens), 1, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def timed(b, plain):
+        ts = []
+        for it in range(reps + 1):
+            ctx.plan(0, b)
+            flush.fill_(it & 1)
+            torch.cuda.synchronize()                # run_plain reads the tile count: keep that wait out of the timing
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            if plain:
+                ctx.run_plain(0)
+            else:
+                ctx.run([0], fuse_combine=False)
+                ctx.combine(0)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * e0.elapsed_time(e1))
+        ctx.check()
+        return _median(ts[1:])
+
+    rows = []
+    op = synth.make_ops(spec)[0]
+    b = ctx.bind(op.cls, op.x.to(dev), torch.from_numpy(op.ids).to(dev), torch.from_numpy(op.w).to(dev), w1, w2)
+    t_pers, y = timed(b, False), b.y.clone()
+    t_plain = timed(b, True)
+    rows.append(dict(case=f"prefill {prefill_tokens} tokens", x_moe=ctx.footprint(0)[0], persistent_us=t_pers, plain_us=t_plain,
+                     same_bits=bool(torch.equal(y, b.y))))
+    x, _ = synth.make_x(spec, decode_tokens, 0, 1)
+    for A in actives:
+        if A < k or A > E:
+            continue
+        ids, w = synth.route_active_pool(np.random.default_rng([seed, A]), decode_tokens, k, E, A)
+        b = ctx.bind(synth.DECODE, x.to(dev), torch.from_numpy(ids).to(dev), torch.from_numpy(w).to(dev), w1, w2)
+        t_pers, y = timed(b, False), b.y.clone()
+        t_plain = timed(b, True)
+        rows.append(dict(case=f"decode {decode_tokens} tokens, {A} active experts", x_moe=ctx.footprint(0)[0],
+                         persistent_us=t_pers, plain_us=t_plain, same_bits=bool(torch.equal(y, b.y))))
+    return rows
+
+
 def main():
+    import sys
+    if "--overhead" in sys.argv:
+        rows = scheduler_overhead()
+        for r in rows:
+            print("%-42s x_moe %4d  persistent %8.1f us  plain launches %8.1f us  (%+.1f %%, %+.1f us)" %
+                  (r["case"], r["x_moe"], r["persistent_us"], r["plain_us"],
+                   100.0 * (r["persistent_us"] / r["plain_us"] - 1.0), r["persistent_us"] - r["plain_us"]))
+        print(json.dumps(rows))
+        return
     rows = study()
     for r in rows:
         print("%-10s q=%-4s prefill done %9.1f us   decode done %9.1f us" %

@@ -201,3 +201,33 @@ def test_sharing_study_runs_and_launch_granularity_sharing_serialises():
     assert all(r["prefill_us"] > 0 and r["decode_us"] > 0 for r in rows)
     assert by[("streams", None)]["decode_us"] > by[("exclusive", None)]["prefill_us"] * 0.9
     assert by[("apk", 96)]["decode_us"] < by[("apk", 96)]["prefill_us"]
+
+
+def test_plain_launches_give_the_same_bits_as_the_persistent_kernel():
+    """moe_run_plain runs the op's gate/up and down tiles as two plain launches (one claiming unit per queue
+    entry, no queue, no budget): the same tile code, so y is bit-identical to the persistent launch; the
+    scheduling-overhead study compares the two on a small shape."""
+    W = weights_to(synth.make_weights(SPEC))
+    ops = synth.make_ops(SPEC)
+    ctx = make_ctx(SPEC, max_tokens=4096, max_ops=2, tile_log_entries=1 << 15)
+    for s_, op in enumerate(ops):
+        b = bind_ops(ctx, [op], W)[0]
+        ctx.plan(s_, b)
+        ctx.run([s_], fuse_combine=True)
+        ctx.check()
+        y = b.y.clone()
+        b.y.fill_(float("nan"))
+        ctx.run_plain(s_)
+        ctx.check()
+        assert torch.equal(y, b.y)
+        log = ctx.tile_log()                   # the log of the last launch: the down tiles, each exactly once
+        assert (log["kind"] == 1).all() and len(np.unique(log["tile"])) == len(log)
+    single = make_ctx(SPEC, max_tokens=4096, max_ops=1, n_ctas=3)          # single-CTA kernel: no plain form
+    b = bind_ops(single, ops[1:], W)[0]
+    single.plan(0, b)
+    with pytest.raises(moe.MoeError):
+        single.run_plain(0)
+    from paper_2607_18002_b200.sharing_study import scheduler_overhead
+    rows = scheduler_overhead(E=32, k=4, H=1024, I=512, prefill_tokens=2048, zipf_s=1.0, decode_tokens=32,
+                              actives=(8, 32), reps=3)
+    assert len(rows) == 3 and all(r["same_bits"] and r["persistent_us"] > 0 and r["plain_us"] > 0 for r in rows)
