@@ -150,13 +150,14 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
  * bounded by wait_limit_us. */
 int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, void* stream);
 
-/* The same tiles as plain (non-persistent) launches, for measuring what the tile scheduler costs
- * (the scheduling-overhead experiment of Section 7.4): one launch for the gate/up tiles of the op in
- * `slot` and one for its down tiles, each with one claiming unit per queue entry -- no queue, no
- * budget, no ready word -- then the stand-alone combine.  Same tile code, bit-identical y.  bf16 on
- * an even grid only (MOE_EINVAL otherwise, and for an op with a ready word or a predecessor).  The
- * grid size is the op's entry count, which lives on the device: this call SYNCHRONISES the stream to
- * read it, so it is a measuring tool, not a serving path. */
+/* The same tiles as a plain (non-persistent) launch, for measuring what the tile scheduler costs
+ * (the scheduling-overhead experiment of Section 7.4): ONE launch with one claiming unit per queue
+ * entry of the op in `slot` -- unit u runs entry u and ends; no queue, no budget, no ready word; a
+ * down tile waits, bounded, for the gate/up tiles of its rows, which belong to units with a lower
+ * index -- then the stand-alone combine.  Same tile code, bit-identical y.  bf16 on an even grid only
+ * (MOE_EINVAL otherwise, and for an op with a ready word or a predecessor).  The grid size is the
+ * op's entry count, which lives on the device: this call SYNCHRONISES the stream to read it, so it
+ * is a measuring tool, not a serving path. */
 int moe_run_plain(moe_ctx_t* ctx, int slot, void* stream);
 
 /* Post-processing: y[t,:] = sum_j w[t,j] * D[flat_to_sorted[t*k+j],:], slots added in

@@ -130,8 +130,8 @@ struct RunArgs {
   int E, k, H, I;
   int dtype, kb_elems;    // MOE_DTYPE_*; K elements per pipeline stage (64 bf16 / 128 e4m3)
   long long wait_ns;
-  int static_kind;        // -1: persistent launch served from the queues.  kGateUp / kDown: a plain launch, one
-                          // claiming unit per queue entry of slots[0], which runs the entry if it is of this kind
+  int static_kind;        // -1: persistent launch served from the queues.  >= 0: a plain launch, claiming unit u
+                          // of the grid runs queue entry u of slots[0] and ends
   int slots[kMaxOps];
 };
 

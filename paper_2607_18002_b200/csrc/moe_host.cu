@@ -359,14 +359,8 @@ int moe_run_plain(moe_ctx_t* ctx, int slot, void* stream) {
   a.kb_elems = kBlockK;
   a.wait_ns = (long long)c.wait_limit_us * 1000;
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
-  if (ps.n_gemm_tiles > 0) {
-    // the down launch starts when the gate/up launch has ended (stream order), so the per-tile dependency
-    // counters it checks are already complete
-    a.static_kind = kGateUp;
-    if (launch_pair(a, ctx->rh(), 2 * ps.n_gemm_tiles, st) != cudaSuccess) return MOE_ECUDA;
-    a.static_kind = kDown;
-    if (launch_pair(a, ctx->rh(), 2 * ps.n_gemm_tiles, st) != cudaSuccess) return MOE_ECUDA;
-  }
+  a.static_kind = 0;
+  if (ps.n_gemm_tiles > 0 && launch_pair(a, ctx->rh(), 2 * ps.n_gemm_tiles, st) != cudaSuccess) return MOE_ECUDA;
   if (launch_combine(ctx->op_dev(slot), ctx->ops[slot].n_tokens, c.top_k, c.hidden, st) != cudaSuccess) return MOE_ECUDA;
   return MOE_OK;
 }

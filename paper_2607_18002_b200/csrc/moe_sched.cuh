@@ -232,15 +232,15 @@ __device__ inline bool wait_op_ready(const Ctx& c, int lane, const TileInfo& ti)
   return true;
 }
 
-// The plain (non-persistent) launch: unit `unit` of the grid takes queue entry `unit` of the run's only op,
-// if that entry is of the launch's kind, and nothing else.  No queue head, no budget, no ready word.
+// The plain (non-persistent) launch: unit `unit` of the grid takes queue entry `unit` of the run's only op
+// and nothing else.  No queue head, no budget, no ready word.  A down tile still waits (bounded) for the
+// gate/up tiles of its rows: they sit earlier in the list, i.e. in units with a lower index.
 __device__ inline void claim_static(const RunArgs* a, int unit, TileInfo& ti) {
   const int slot = a->slots[0];
   const OpDev* op = &a->ops[slot];
   ti.kind = kEnd;
   if (unit >= op->plan->n_gemm_tiles) return;
   const int4 got = op->tile_list[unit];
-  if (entry_kind(got) != a->static_kind) return;
   ti.kind = entry_kind(got);
   ti.n = entry_n(got);
   ti.m = entry_m(got);

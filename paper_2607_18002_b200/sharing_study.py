@@ -134,8 +134,7 @@ def scheduler_overhead(E=256, k=8, H=3072, I=1536, prefill_tokens=8192, zipf_s=1
     """What the persistent kernel's tile scheduling costs against plain launches of the SAME tile code
     (the experiment of Section 7.4): for a prefill-sized op (contiguous layout, Zipf routing) and for a
     decode-sized op over a growing number of active experts, the time of moe_run + moe_combine next to the
-    time of moe_run_plain (one gate/up launch and one down launch with a claiming unit per tile, then the
-    combine).  CUDA events, median of `reps` after one warm-up, L2 flushed between launches.  Returns rows of
+    time of moe_run_plain (one launch with a claiming unit per tile, then the combine).  CUDA events, median of `reps` after one warm-up, L2 flushed between launches.  Returns rows of
     dict(case, x_moe, persistent_us, plain_us)."""
     import torch
 
