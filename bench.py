@@ -133,8 +133,11 @@ def visible_index(local_rank: int) -> int:
 class Workload:
     """Device-resident inputs of one workload plus the calls of one step."""
 
-    def __init__(self, name: str, rank: int, device: torch.device, tile_log: int = 0):
-        """Generates the workload's seeded inputs on the host, uploads them and plans nothing yet."""
+    def __init__(self, name: str, rank: int, device: torch.device, tile_log: int = 0, pair: bool = True):
+        """Generates the workload's seeded inputs on the host, uploads them and plans nothing yet.
+        pair: a co-scheduled decode + prefill op of a layer run in their paired form (moe_plan_pair: decode rows
+        travel in carrier tiles with prefill rows of the same expert, each weight tile is streamed once)."""
+        self.pair = pair
         import paper_2607_18002_b200 as moe
         self.moe = moe
         self.name = name
@@ -152,7 +155,9 @@ class Workload:
         self.fp8 = sh.dtype == "fp8"
         el = 1 if self.fp8 else 2
         self.layers = []
-        self.ctx = moe.Context(sh.E, sh.k, sh.H, sh.I, max(T for _, T in self.spec.ops),
+        # the paired form keeps the rows of both ops in one slot's scratch
+        self.max_tokens = sum(T for _, T in self.spec.ops) if len(self.spec.ops) > 1 else self.spec.ops[0][1]
+        self.ctx = moe.Context(sh.E, sh.k, sh.H, sh.I, self.max_tokens,
                                max_ops=len(self.spec.ops), tile_log_entries=tile_log,
                                dtype=moe.MOE_DTYPE_FP8_E4M3 if self.fp8 else moe.MOE_DTYPE_BF16,
                                device=device)
@@ -188,16 +193,31 @@ class Workload:
                 self.bytes_alg += float(active.sum()) * 3 * (sh.H // 128) * (sh.I // 128) * 4
             self.layers.append((ops, bound, host))
         self.launches_per_step = sum(sum(plan_kernels(o.T, sh.k, sh.E) for o in ops_) + 1 + (1 if self.spec.layers > 1 else 0)
-                                     for ops_, _, _ in self.layers)
+                                     + (2 if self._pairs(ops_) else 0) for ops_, _, _ in self.layers)
+
+    def _pairs(self, ops):
+        """(prefill slot, decode slot) of a layer that runs paired, else None."""
+        if not self.pair or len(ops) != 2:
+            return None
+        cls = [o.cls for o in ops]
+        if sorted(cls) != [synth.DECODE, synth.PREFILL]:
+            return None
+        return cls.index(synth.PREFILL), cls.index(synth.DECODE)
+
+    def plan_layer(self, ctx, ops, bound):
+        for s, b in enumerate(bound):
+            ctx.plan(s, b)
+        pr = self._pairs(ops)
+        if pr:
+            ctx.plan_pair(pr[0], pr[1], 0)
 
     def step(self, ev=None):
         """Whole hot path for one batch; ev (optional) collects (before_run, after_run) events."""
         ctx = self.ctx
-        for li, (_, bound, _) in enumerate(self.layers):
+        for li, (ops, bound, _) in enumerate(self.layers):
             if self.spec.layers > 1:
                 ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
-            for s, b in enumerate(bound):
-                ctx.plan(s, b)
+            self.plan_layer(ctx, ops, bound)
             if ev is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
                 e0.record()
@@ -214,7 +234,7 @@ class Workload:
             return
         moe, sh, device = self.moe, self.sh, self.device
         dev = lambda t: None if t is None else t.to(device)
-        self.ctx2 = moe.Context(sh.E, sh.k, sh.H, sh.I, max(T for _, T in self.spec.ops),
+        self.ctx2 = moe.Context(sh.E, sh.k, sh.H, sh.I, self.max_tokens,
                                 max_ops=len(self.spec.ops),
                                 dtype=moe.MOE_DTYPE_FP8_E4M3 if self.fp8 else moe.MOE_DTYPE_BF16, device=device)
         n_sets = len(self.W)
@@ -234,7 +254,7 @@ class Workload:
         copies cost when they are not hidden behind the neighbouring steps' kernels."""
         ctx = self.ctx
         for _ in range(steps):
-            for li, (_, bound, host) in enumerate(self.layers):
+            for li, (ops, bound, host) in enumerate(self.layers):
                 for b, (hx, hi, hw, hy, hs) in zip(bound, host):
                     b.x.copy_(hx, non_blocking=True)
                     if hs is not None:
@@ -243,8 +263,7 @@ class Workload:
                     b.topk_w.copy_(hw, non_blocking=True)
                 if self.spec.layers > 1:
                     ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
-                for s_, b in enumerate(bound):
-                    ctx.plan(s_, b)
+                self.plan_layer(ctx, ops, bound)
                 ctx.run(list(range(len(bound))), fuse_combine=True)
                 for b, (_, _, _, hy, _) in zip(bound, host):
                     hy.copy_(b.y, non_blocking=True)
@@ -260,7 +279,7 @@ class Workload:
         free = {}
         for step in range(steps):
             ctx, layers = sets[step % 2]
-            for li, (_, bound, host) in enumerate(layers):
+            for li, (ops_l, bound, host) in enumerate(layers):
                 key = (step % 2, li)
                 with torch.cuda.stream(self.s_h2d):
                     if key in free:
@@ -277,8 +296,7 @@ class Workload:
                     self.s_comp.wait_event(e_in)
                     if self.spec.layers > 1:
                         ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
-                    for s_, b in enumerate(bound):
-                        ctx.plan(s_, b)
+                    self.plan_layer(ctx, ops_l, bound)
                     ctx.run(list(range(len(bound))), fuse_combine=True)
                     e_run = torch.cuda.Event()
                     e_run.record(self.s_comp)
@@ -396,29 +414,40 @@ def tile_stats(w: Workload):
         w.step()
         ctx.check()
         return {"corun": _log_summary(ctx.tile_log())}
-    out = {"per_budget": {}}
-    budgets = synth.C4_BUDGETS if w.spec.layers > 1 else (None,)
+    out = {"per_budget": {}, "paired": bool(w.pair)}
+    # the workload's own budgets, then larger ones: the latency of a decode op that streams most experts'
+    # weights follows its share of the SMs (and with it of the HBM bandwidth)
+    own = tuple(synth.C4_BUDGETS) if w.spec.layers > 1 else (None,)
+    budgets = own + ((96, 112, 128) if w.spec.layers > 1 else ())
     pooled = {"co": [], "iso": []}
-    for li, q in enumerate(budgets):
-        if li >= len(w.layers):
-            break
-        _, bound, _ = w.layers[li]
+    for bi, q in enumerate(budgets):
+        li = bi % len(w.layers)
+        ops, bound, _ = w.layers[li]
         dec = [s for s, b in enumerate(bound) if b.c.cls == 0]
         if q is not None:
             ctx.set_budget(q)
-        for s, b in enumerate(bound):
-            ctx.plan(s, b)
+        w.plan_layer(ctx, ops, bound)
         ctx.run(list(range(len(bound))), fuse_combine=True)
         ctx.check()
         log_co = ctx.tile_log()
         co = _log_summary(log_co)
-        ctx.run(dec, fuse_combine=True)
+        ctx.run(dec, fuse_combine=True)           # one op of a pair alone: the plain form runs
         ctx.check()
         log_iso = ctx.tile_log()
         iso = _log_summary(log_iso)
         entry = {"layer": li, "corun": co, "decode_isolated": iso}
         entry.update(_ratios(co, iso))
+        if w.pair:                                 # the same launch without pairing, for comparison
+            for s, b in enumerate(bound):
+                ctx.plan(s, b)
+            ctx.run(list(range(len(bound))), fuse_combine=True)
+            ctx.check()
+            un = _log_summary(ctx.tile_log())
+            entry["unpaired"] = {"kernel_span_us": un["kernel_span_us"], "decode_op_us": un["decode_op_us"],
+                                 "decode_op_ratio": un["decode_op_us"] / iso["decode_op_us"]}
         out["per_budget"][str(q)] = entry
+        if q not in own:
+            continue                               # the pooled percentiles are over the workload's own budgets
         for key, lg in (("co", log_co), ("iso", log_iso)):
             m = (lg["cls"] == 0) & (lg["kind"] < 2)
             t0 = int(lg["t_claim"].min())
@@ -432,6 +461,10 @@ def tile_stats(w: Workload):
                                          "isolated_p50": float(np.percentile(iso[i], 50)),
                                          "isolated_p99": float(np.percentile(iso[i], 99))}
     out["decode_op_ratio"] = {q: e["decode_op_ratio"] for q, e in out["per_budget"].items() if "decode_op_ratio" in e}
+    out["decode_tile_latency_p99_ratio_by_budget"] = {q: e["decode_tile_latency_p99_ratio"] for q, e in out["per_budget"].items()
+                                                      if "decode_tile_latency_p99_ratio" in e}
+    within = [int(q) for q, r in out["decode_tile_latency_p99_ratio_by_budget"].items() if q != "None" and r <= 1.3]
+    out["smallest_budget_with_latency_p99_within_1.3x"] = min(within) if within else None
     out["readings"] = ("service = commit - claim of a decode tile; latency = commit - launch start (all ops ready at "
                        "launch); isolated = the same decode op alone in the launch at the same budget")
     _, bound, _ = w.layers[min(1, len(w.layers) - 1)]
@@ -581,7 +614,7 @@ def measure(name: str, args, K: int, Wm: int, rank: int, world: int, local: int,
     every persistent launch for the roofline, optionally the end-to-end loops with host buffers and the
     tile-log statistics.  Returns the fields of a bench line."""
     from paper_2607_18002_b200 import dist
-    w = Workload(name, rank, device, tile_log=(1 << 17) if tile_log else 0)
+    w = Workload(name, rank, device, tile_log=(1 << 17) if tile_log else 0, pair=not args.no_pair)
     for _ in range(Wm):
         w.step()
     w.ctx.check()
@@ -677,7 +710,8 @@ def measure(name: str, args, K: int, Wm: int, rank: int, world: int, local: int,
                       "inter": sh.I, "l2": "inputs_exceed_l2 (weights >> 126 MB, no flush)",
                       "buffers": "the same X / y buffers every step: the step's 7-10 GB of weights pass through "
                                  "the 126 MB L2 between two uses of a buffer",
-                      "replicas": world, "fused_combine": True},
+                      "replicas": world, "fused_combine": True,
+                      "paired_ops": bool(w.pair and any(w._pairs(o) for o, _, _ in w.layers))},
            "clocks": clk.summary(), "gpu_launches": w.launches_per_step * K, "roofline": roof}
     if e2e_out:
         res["e2e"], res["e2e_serial"] = e2e_out, e2e_serial
@@ -737,6 +771,8 @@ def main():
     ap.add_argument("--tile-log", action="store_true", help="add per-tile timing statistics of one extra untimed step")
     ap.add_argument("--one-launch", action="store_true",
                     help="multi-layer workloads: also time all layers as one persistent launch per step")
+    ap.add_argument("--no-pair", action="store_true",
+                    help="co-scheduled workloads: run the decode and the prefill op unpaired (no carrier tiles)")
     ap.add_argument("--no-sub", action="store_true",
                     help="default workload only: skip the c2 / c4 / c5 sub-results")
     args = ap.parse_args()

@@ -150,6 +150,22 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream);
  * bounded by wait_limit_us. */
 int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, void* stream);
 
+/* Pairs a prefill op and a decode op that share their expert weights (both planned, same w_gate_up /
+ * w_down / scale pointers) so that a launch running both streams an expert's weight tile ONCE for rows of
+ * both: the decode op's rows of an expert travel in "carrier" tiles together with as many of that expert's
+ * prefill rows as fit into the decode rows' last tile of `carrier_rows` rows (128, or 256 for bf16; 0 = the
+ * largest).  Carrier tiles belong to the decode class -- decode priority and the budget work as before
+ * (Sections 4.2, 6.4) -- and the prefill op keeps the remaining rows.  A row's arithmetic does not depend
+ * on the tile it sits in, so y of both ops is bit-identical to the unpaired launch; counts, offsets and the
+ * permutations of moe_plan are untouched (the shared row space is private workspace).
+ *   - call after moe_plan of both slots, on the same stream; a later moe_plan of either slot ends the pairing;
+ *   - moe_run uses the paired form when BOTH slots are in the launch, the plain form otherwise;
+ *   - the prefill op is complete (done word, successors, its combine tiles) only when the decode op's GEMM
+ *     tiles are, because some of them carry its rows: a decode op that never becomes ready holds it back;
+ *   - n_tokens of both ops together must fit max_tokens_per_op (the shared row space lives in one slot's
+ *     scratch), else MOE_ENOSPC; both ops need at least one token (MOE_EINVAL). */
+int moe_plan_pair(moe_ctx_t* ctx, int slot_prefill, int slot_decode, int carrier_rows, void* stream);
+
 /* The same tiles as a plain (non-persistent) launch, for measuring what the tile scheduler costs
  * (the scheduling-overhead experiment of Section 7.4): ONE launch with one claiming unit per queue
  * entry of the op in `slot` -- unit u runs entry u and ends; no queue, no budget, no ready word; a

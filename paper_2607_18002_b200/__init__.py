@@ -29,7 +29,7 @@ MOE_TILE_M = 128
 EXPORTS = ("moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_run",
            "moe_combine", "moe_set_budget", "moe_set_budget_scaled", "moe_get_budget", "moe_status", "moe_footprint",
            "moe_read_tile_table", "moe_read_tile_log", "moe_sm_count", "moe_ctas_per_tile", "moe_strerror",
-           "moe_plan_static", "moe_route", "moe_run_plain")
+           "moe_plan_static", "moe_route", "moe_run_plain", "moe_plan_pair")
 MOE_PLAN_STATIC_MAX_ROWS, MOE_PLAN_STATIC_MAX_EXPERTS = 32768, 256
 
 
@@ -90,6 +90,7 @@ def lib() -> C.CDLL:
         L.moe_run.argtypes = [vp, C.POINTER(i32), C.c_int, C.c_int, vp]
         L.moe_combine.argtypes = [vp, C.c_int, vp]
         L.moe_run_plain.argtypes = [vp, C.c_int, vp]
+        L.moe_plan_pair.argtypes = [vp, C.c_int, C.c_int, C.c_int, vp]
         L.moe_set_budget.argtypes = [vp, C.c_int, vp]
         L.moe_set_budget_scaled.argtypes = [vp, C.c_int, C.c_int, C.c_double, C.c_int, vp]
         L.moe_get_budget.argtypes = [vp, C.POINTER(i32)]
@@ -146,6 +147,11 @@ def moe_run(ctx: int, slots: Sequence[int], fuse_combine: bool, stream: int) -> 
     arr = (C.c_int32 * len(slots))(*slots)
     _check(lib().moe_run(C.c_void_p(ctx), arr, len(slots), int(bool(fuse_combine)),
                          C.c_void_p(stream)), "moe_run")
+
+
+def moe_plan_pair(ctx: int, slot_prefill: int, slot_decode: int, carrier_rows: int, stream: int) -> None:
+    _check(lib().moe_plan_pair(C.c_void_p(ctx), slot_prefill, slot_decode, carrier_rows, C.c_void_p(stream)),
+           "moe_plan_pair")
 
 
 def moe_run_plain(ctx: int, slot: int, stream: int) -> None:
@@ -328,6 +334,9 @@ class Context:
 
     def run(self, slots: Sequence[int], fuse_combine: bool = False, stream=None):
         moe_run(self.ctx, list(slots), fuse_combine, self._stream(stream))
+
+    def plan_pair(self, slot_prefill: int, slot_decode: int, carrier_rows: int = 0, stream=None):
+        moe_plan_pair(self.ctx, slot_prefill, slot_decode, carrier_rows, self._stream(stream))
 
     def run_plain(self, slot: int, stream=None):
         moe_run_plain(self.ctx, slot, self._stream(stream))

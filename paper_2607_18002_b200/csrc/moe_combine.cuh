@@ -1,4 +1,4 @@
-// Router-weighted combine (post-processing): y[t,:] = sum_j w[t,j] * D[flat_to_sorted[t*k+j],:]
+// Router-weighted combine (post-processing): y[t,:] = sum_j w[t,j] * D[row(t,j),:], row = flat_to_sorted[t*k+j]
 // with the k slots added in order in fp32 (the last step of the MoE module of Section 2.1 of the
 // paper).  One device routine serves the stand-alone kernel and the combine tiles of the
 // persistent kernel.  A permutation entry outside [0, T*k) -- left by a plan that rejected an
@@ -31,18 +31,18 @@ __device__ __forceinline__ void combine_add4(float (&acc)[8], const uint4 (&d)[4
   }
 }
 
-__device__ __forceinline__ int f2s_entry(const OpDev* op, int i) { return op->flat_to_sorted[i]; }
+__device__ __forceinline__ int f2s_entry(const OpDev* op, int i) { return op->comb_index[i]; }
 
 __device__ __noinline__ inline void combine_tokens(const OpDev* op, int t0, int t1, int k, int H, int tid,
                                                    int nthr) {
-  const unsigned n_rows = (unsigned)op->n_rows;
+  const unsigned n_rows = (unsigned)op->space_rows;    // rows of the packed space D lives in
   // every permutation entry of these tokens is checked once, ahead of the loops that use them
   for (int i = t0 * k + tid; i < t1 * k; i += nthr)
     if ((unsigned)f2s_entry(op, i) >= n_rows) report(op->status, MOE_EBOUNDS, i / k, i % k, f2s_entry(op, i), 2);
   const int vec_per_row = H / 8;
   const uint4* D = reinterpret_cast<const uint4*>(op->D);
   uint4* y = reinterpret_cast<uint4*>(op->y);
-  const int* f2s = op->flat_to_sorted;
+  const int* f2s = op->comb_index;
   const float* w = op->topk_w;
   const int total = (t1 - t0) * vec_per_row;
   if (k <= 8 && nthr >= 16 && vec_per_row % 16 == 0) {

@@ -46,6 +46,8 @@ struct PlanState {
   int n_gemm_tiles;   // queue entries of kind gate/up or down
   int n_comb_tiles;   // queue entries of kind combine (follow the GEMM entries)
   int planned;        // 1 after a moe_plan that accepted every expert id, else 0
+  int n_extra_gemm;   // paired prefill op: GEMM entries of the decode op's list that carry rows of this op
+  int pad[3];
 };
 
 // Zeroed by moe_run before every launch.
@@ -97,7 +99,18 @@ struct __align__(128) OpDev {
   RunState* run;
   int* g1_done;          // [max_mtiles] committed gate/up tiles per work tile
   Status* status;        // the context's device status block
+  // Which list of routed rows the run kernels walk.  A plain op: its own permutation (the plan's public
+  // outputs).  The paired form of a decode + prefill op that share their weights (moe_plan_pair): one row
+  // space for both, every entry of the gather list tagged with the slot whose row it is.
+  const int* gather_list;   // packed row -> flat routed index (paired: | slot << kRowSlotShift)
+  const int* comb_index;    // flat routed index -> packed row of D
+  int space_rows;           // rows of the packed space that A, D and comb_index refer to
+  int paired;               // 1: this is the paired form of the slot
+  int partner;              // paired: descriptor index of the other op of the pair, else -1
+  int pad_[3];
 };
+constexpr int kRowSlotShift = 27;                       // a flat routed index stays below 2^27 (moe_create checks)
+constexpr int kRowFlatMask = (1 << kRowSlotShift) - 1;
 
 struct Status {   // first error wins (atomicCAS on code)
   int code;
@@ -130,10 +143,14 @@ struct RunArgs {
   int E, k, H, I;
   int dtype, kb_elems;    // MOE_DTYPE_*; K elements per pipeline stage (64 bf16 / 128 e4m3)
   long long wait_ns;
+  int n_slots;            // slots of the context; descriptor d >= n_slots is the paired form of slot d - n_slots
+  signed char desc[kMaxOps];   // slot -> the descriptor that stands for it in this launch
   int static_kind;        // -1: persistent launch served from the queues.  >= 0: a plain launch, claiming unit u
                           // of the grid runs queue entry u of slots[0] and ends
-  int slots[kMaxOps];
+  int slots[kMaxOps];     // descriptor indices of the launch's ops, in the order given
 };
+
+__device__ __forceinline__ int slot_of(const RunArgs* a, int desc) { return desc >= a->n_slots ? desc - a->n_slots : desc; }
 
 __device__ __noinline__ inline void report(Status* st, int code, int d0, int d1, int d2, int d3) {
   if (atomicCAS(&st->code, 0, code) == 0) {

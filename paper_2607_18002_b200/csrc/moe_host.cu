@@ -11,6 +11,9 @@
 namespace moe {
 cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, int E, int NT1,
                         int NT2, int work_rows, cudaStream_t stream);
+cudaError_t launch_plan_pair(const OpDev* dp, const OpDev* pp, const OpDev* d, const OpDev* p, int* gather_m, int* comb_d,
+                             int* comb_p, int Rd, int Rp, int E, int NT1, int NT2, int work_rows, int carrier_rows,
+                             int slot_d, int slot_p, cudaStream_t stream);
 cudaError_t launch_combine(const OpDev* d_op, int T, int k, int H, cudaStream_t stream);
 cudaError_t prepare_run_kernel();
 cudaError_t launch_run(const RunArgs& args, RunHead* rh, int n_ctas, cudaStream_t stream);
@@ -29,6 +32,7 @@ struct Layout {
   size_t global_off, ops_off, runzero_off, runzero_bytes, log_off, slots_off, slot_stride;
   // inside a slot
   size_t A_off, D_off, mtiles_off, tiles_off, hist_off, plan_off;
+  size_t ptiles_off, pgather_off, pcomb_off, pplan_off;   // paired form: queue list, shared-space permutation, plan state
   // inside the run-zero region (after RunHead)
   size_t rs_stride;      // RunState + g1_done[max_mtiles], per slot
   size_t total;
@@ -45,7 +49,8 @@ int check_config(const moe_config_t* c) {
   if (c->inter / kTileN1 > 255 || c->hidden / kTileN2 > 255) return MOE_EINVAL;
   if (c->dtype != MOE_DTYPE_BF16 && c->dtype != MOE_DTYPE_FP8_E4M3) return MOE_EINVAL;
   if (c->max_tokens_per_op < 1 || c->max_ops < 1 || c->max_ops > kMaxOps) return MOE_EINVAL;
-  if ((long long)c->max_tokens_per_op * c->top_k > (1 << 20) * (long long)kTileM) return MOE_EINVAL;
+  // a flat routed index must fit below bit kRowSlotShift (the paired form tags it with a slot above that)
+  if ((long long)c->max_tokens_per_op * c->top_k >= (1ll << kRowSlotShift)) return MOE_EINVAL;
   // the combine addresses the rows of the down-GEMM output by 32-bit offsets in 16-byte units
   if ((long long)c->max_tokens_per_op * c->top_k * (c->hidden / 8) >= (1ll << 32)) return MOE_EINVAL;
   if (c->wait_limit_us < 0 || c->tile_log_entries < 0 || c->n_ctas < 0) return MOE_EINVAL;
@@ -70,11 +75,15 @@ Layout make_layout(const moe_config_t* c) {
   L.tiles_off = off;   off = align_up(off + (size_t)L.max_tiles * sizeof(int4), 1024);
   L.hist_off = off;    off = align_up(off + 2 * n_chunks * E * 4, 1024);   // histogram + base ranks
   L.plan_off = off;    off = align_up(off + sizeof(PlanState), 1024);
+  L.ptiles_off = off;  off = align_up(off + (size_t)L.max_tiles * sizeof(int4), 1024);
+  L.pgather_off = off; off = align_up(off + (size_t)L.max_rows * 4, 1024);
+  L.pcomb_off = off;   off = align_up(off + (size_t)L.max_rows * 4, 1024);
+  L.pplan_off = off;   off = align_up(off + sizeof(PlanState), 1024);
   L.slot_stride = off;
 
   size_t g = 0;
   L.global_off = g;    g = align_up(g + sizeof(Global), 1024);
-  L.ops_off = g;       g = align_up(g + sizeof(OpDev) * c->max_ops, 1024);
+  L.ops_off = g;       g = align_up(g + sizeof(OpDev) * 2 * c->max_ops, 1024);   // plain and paired descriptors
   L.runzero_off = g;
   L.rs_stride = align_up(sizeof(RunState) + (size_t)L.max_mtiles * 4, 16);
   L.runzero_bytes = align_up(sizeof(RunHead) + L.rs_stride * c->max_ops, 1024);
@@ -103,6 +112,10 @@ struct moe_ctx {
   bool planned[kMaxOps];
   OpDev host_ops[kMaxOps];      // what the device copy of each slot holds (tensor maps included)
   bool uploaded[kMaxOps];
+  OpDev host_pair[kMaxOps];     // what the device copy of each slot's paired descriptor holds
+  bool pair_uploaded[kMaxOps];
+  int pair_of[kMaxOps];         // slot paired with this one by moe_plan_pair since both were last planned, or -1
+  bool ran_paired[kMaxOps];     // the slot's last moe_run used its paired form (moe_combine follows it)
   Global* g() const { return reinterpret_cast<Global*>(ws + L.global_off); }
   RunHead* rh() const { return reinterpret_cast<RunHead*>(ws + L.runzero_off); }
   unsigned char* slot_base(int s) const { return ws + L.slots_off + L.slot_stride * s; }
@@ -203,10 +216,15 @@ int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_c
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   memset(ctx->planned, 0, sizeof(ctx->planned));
   memset(ctx->uploaded, 0, sizeof(ctx->uploaded));
+  memset(ctx->ran_paired, 0, sizeof(ctx->ran_paired));
+  memset(ctx->pair_uploaded, 0, sizeof(ctx->pair_uploaded));
+  for (int s = 0; s < kMaxOps; ++s) ctx->pair_of[s] = -1;
   // zero the control blocks (status, budget, run state, plan states)
   cudaError_t e = cudaMemset(ctx->ws, 0, L.slots_off);
-  for (int s = 0; s < cfg->max_ops && e == cudaSuccess; ++s)
+  for (int s = 0; s < cfg->max_ops && e == cudaSuccess; ++s) {
     e = cudaMemset(ctx->slot_base(s) + L.plan_off, 0, sizeof(PlanState));
+    if (e == cudaSuccess) e = cudaMemset(ctx->slot_base(s) + L.pplan_off, 0, sizeof(PlanState));
+  }
   if (e != cudaSuccess) { delete ctx; return MOE_ECUDA; }
   *out = ctx;
   return MOE_OK;
@@ -262,6 +280,15 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   h.run = reinterpret_cast<RunState*>(ctx->rs_base(slot));
   h.g1_done = reinterpret_cast<int*>(ctx->rs_base(slot) + sizeof(RunState));
   h.status = &ctx->g()->status;
+  h.gather_list = op->sorted_to_flat;
+  h.comb_index = op->flat_to_sorted;
+  h.space_rows = h.n_rows;
+  h.paired = 0;
+  h.partner = -1;
+  // a new plan for the slot ends any pairing it was part of
+  if (ctx->pair_of[slot] >= 0) ctx->pair_of[ctx->pair_of[slot]] = -1;
+  ctx->pair_of[slot] = -1;
+  ctx->ran_paired[slot] = false;
   // Re-planning a slot with the same buffers (the usual serving loop) reuses the descriptors
   // already on the device: encoding seven tensor maps and uploading them is host time.
   const bool same = ctx->uploaded[slot] && memcmp(&ctx->ops[slot], op, sizeof(moe_op_t)) == 0;
@@ -305,6 +332,19 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
     if (!ctx->planned[s]) return MOE_ENOTPLANNED;
     for (int j = 0; j < i; ++j) if (slots[j] == s) return MOE_EINVAL;
     a.slots[i] = s;
+  }
+  // a slot whose pair partner is in the same launch runs in its paired form
+  a.n_slots = c.max_ops;
+  for (int s = 0; s < kMaxOps; ++s) a.desc[s] = (signed char)s;
+  for (int i = 0; i < n_ops; ++i) {
+    const int s = slots[i], q = ctx->pair_of[s];
+    bool both = false;
+    for (int j = 0; j < n_ops && q >= 0; ++j) both |= slots[j] == q;
+    ctx->ran_paired[s] = both;
+    if (both) {
+      a.slots[i] = c.max_ops + s;
+      a.desc[s] = (signed char)(c.max_ops + s);
+    }
   }
   for (int i = 0; i < n_ops; ++i) {      // after_op must name an op of this run
     const int dep = ctx->ops[slots[i]].after_op;
@@ -358,6 +398,9 @@ int moe_run_plain(moe_ctx_t* ctx, int slot, void* stream) {
   a.dtype = c.dtype;
   a.kb_elems = kBlockK;
   a.wait_ns = (long long)c.wait_limit_us * 1000;
+  a.n_slots = c.max_ops;
+  for (int s = 0; s < kMaxOps; ++s) a.desc[s] = (signed char)s;
+  ctx->ran_paired[slot] = false;
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
   a.static_kind = 0;
   if (ps.n_gemm_tiles > 0 && launch_pair(a, ctx->rh(), 2 * ps.n_gemm_tiles, st) != cudaSuccess) return MOE_ECUDA;
@@ -368,9 +411,69 @@ int moe_run_plain(moe_ctx_t* ctx, int slot, void* stream) {
 int moe_combine(moe_ctx_t* ctx, int slot, void* stream) {
   if (!ctx || slot < 0 || slot >= ctx->cfg.max_ops) return MOE_EINVAL;
   if (!ctx->planned[slot]) return MOE_ENOTPLANNED;
-  if (launch_combine(ctx->op_dev(slot), ctx->ops[slot].n_tokens, ctx->cfg.top_k, ctx->cfg.hidden,
+  // after a launch that ran the slot in its paired form, the expert outputs lie in the pair's shared row space
+  const int desc = ctx->ran_paired[slot] ? ctx->cfg.max_ops + slot : slot;
+  if (launch_combine(ctx->op_dev(desc), ctx->ops[slot].n_tokens, ctx->cfg.top_k, ctx->cfg.hidden,
                      static_cast<cudaStream_t>(stream)) != cudaSuccess)
     return MOE_ECUDA;
+  return MOE_OK;
+}
+
+int moe_plan_pair(moe_ctx_t* ctx, int slot_prefill, int slot_decode, int carrier_rows, void* stream) {
+  if (!ctx) return MOE_EINVAL;
+  const moe_config_t& c = ctx->cfg;
+  const int sp = slot_prefill, sd = slot_decode;
+  if (sp < 0 || sp >= c.max_ops || sd < 0 || sd >= c.max_ops || sp == sd) return MOE_EINVAL;
+  if (!ctx->planned[sp] || !ctx->planned[sd]) return MOE_ENOTPLANNED;
+  const moe_op_t &op = ctx->ops[sp], &od = ctx->ops[sd];
+  if (op.cls != MOE_CLASS_PREFILL || od.cls != MOE_CLASS_DECODE) return MOE_EINVAL;
+  // one weight tile can only serve rows of both ops if both ops read the same weights
+  if (op.w_gate_up != od.w_gate_up || op.w_down != od.w_down || op.s_gate_up != od.s_gate_up || op.s_down != od.s_down)
+    return MOE_EINVAL;
+  const bool fp8 = c.dtype == MOE_DTYPE_FP8_E4M3;
+  if (carrier_rows == 0) carrier_rows = fp8 ? kWorkRowsFp8 : kWorkRowsBf16;
+  if (carrier_rows != 128 && !(carrier_rows == 256 && !fp8)) return MOE_EINVAL;
+  const Layout& L = ctx->L;
+  const long long Rp = (long long)op.n_tokens * c.top_k, Rd = (long long)od.n_tokens * c.top_k;
+  if (Rp + Rd > L.max_rows) return MOE_ENOSPC;      // the shared row space lives in one slot's scratch
+  if (op.n_tokens == 0 || od.n_tokens == 0) return MOE_EINVAL;
+  unsigned char *bp = ctx->slot_base(sp), *bd = ctx->slot_base(sd);
+  int* gather_m = reinterpret_cast<int*>(bp + L.pgather_off);
+  OpDev hp = ctx->host_ops[sp], hd = ctx->host_ops[sd];
+  // both paired descriptors address the prefill slot's scratch (A, its scales, D) as the shared row space
+  hd.A = hp.A; hd.a_scale = hp.a_scale; hd.D = hp.D;
+  hd.tm_a8 = hp.tm_a8; hd.tm_a32 = hp.tm_a32; hd.tm_a128 = hp.tm_a128; hd.tm_a256 = hp.tm_a256;
+  OpDev* both[2] = {&hp, &hd};
+  for (int i = 0; i < 2; ++i) {
+    OpDev* h = both[i];
+    unsigned char* b = i == 0 ? bp : bd;
+    h->tile_list = reinterpret_cast<int4*>(b + L.ptiles_off);
+    h->plan = reinterpret_cast<PlanState*>(b + L.pplan_off);
+    h->gather_list = gather_m;
+    h->comb_index = reinterpret_cast<int*>(b + L.pcomb_off);
+    h->space_rows = (int)(Rp + Rd);
+    h->paired = 1;
+    h->partner = c.max_ops + (i == 0 ? sd : sp);
+  }
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // the usual loop pairs the same two ops on the same buffers again and again: upload only what changed
+  const int which[2] = {sp, sd};
+  for (int i = 0; i < 2; ++i) {
+    const int s = which[i];
+    if (ctx->pair_uploaded[s] && memcmp(&ctx->host_pair[s], both[i], sizeof(OpDev)) == 0) continue;
+    write_op_kernel<<<1, 128, 0, st>>>(*both[i], ctx->op_dev(c.max_ops + s));
+    if (cudaGetLastError() != cudaSuccess) { ctx->pair_uploaded[s] = false; return MOE_ECUDA; }
+    ctx->host_pair[s] = *both[i];
+    ctx->pair_uploaded[s] = true;
+  }
+  if (launch_plan_pair(ctx->op_dev(c.max_ops + sd), ctx->op_dev(c.max_ops + sp), ctx->op_dev(sd), ctx->op_dev(sp), gather_m,
+                       reinterpret_cast<int*>(bd + L.pcomb_off), reinterpret_cast<int*>(bp + L.pcomb_off), (int)Rd, (int)Rp,
+                       c.n_experts, L.NT1, L.NT2, fp8 ? kWorkRowsFp8 : kWorkRowsBf16, carrier_rows, sd, sp, st) != cudaSuccess)
+    return MOE_ECUDA;
+  if (ctx->pair_of[sp] >= 0) ctx->pair_of[ctx->pair_of[sp]] = -1;
+  if (ctx->pair_of[sd] >= 0) ctx->pair_of[ctx->pair_of[sd]] = -1;
+  ctx->pair_of[sp] = sd;
+  ctx->pair_of[sd] = sp;
   return MOE_OK;
 }
 
@@ -411,7 +514,12 @@ int moe_status(moe_ctx_t* ctx, int32_t* code, int32_t detail[4]) {
   *code = s.code;
   if (detail) for (int i = 0; i < 4; ++i) detail[i] = s.detail[i];
   // a plan that met an expert id out of range left its slot without a usable permutation
-  if (s.code == MOE_EBADID && s.detail[0] >= 0 && s.detail[0] < ctx->cfg.max_ops) ctx->planned[s.detail[0]] = false;
+  if (s.code == MOE_EBADID && s.detail[0] >= 0 && s.detail[0] < ctx->cfg.max_ops) {
+    const int bad = s.detail[0];
+    ctx->planned[bad] = false;
+    if (ctx->pair_of[bad] >= 0) ctx->pair_of[ctx->pair_of[bad]] = -1;
+    ctx->pair_of[bad] = -1;
+  }
   if (s.code != 0 || s.abort != 0)
     if (cudaMemset(&ctx->g()->status, 0, sizeof(Status)) != cudaSuccess) return MOE_ECUDA;
   return MOE_OK;

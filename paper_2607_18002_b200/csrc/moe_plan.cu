@@ -81,16 +81,99 @@ __device__ inline int block_excl_scan(int v, int* total, int* warp_sums) {
   return res;
 }
 
+// ---------------------------------------------------------------- the ordered tile list of one op
+// Shared-memory scratch of build_tile_list (one block of 1024 threads).
+struct ListScratch {
+  int warp_sums[33];
+  int work[kMaxExperts], grp[kMaxExperts], moff[kMaxExperts], w0[kMaxExperts];
+  int g_cnt[kMaxExperts], g_base1[kMaxExperts], g_base2[kMaxExperts];
+  int ntiles;
+};
+
+// Writes the queue list of an op whose expert e holds rows [off[e], off[e] + cnt[e]) of the packed row space
+// (cnt / off in shared memory), and its PlanState.
+// Work tiles (the unit the queues hand out): up to `work_rows` consecutive rows of one
+// expert, i.e. one or two adjacent m-tiles that share each weight tile they read.
+// Dependency groups: consecutive experts holding at least kGroupWork work tiles.  The list
+// is  G1(g0) G1(g1) G2(g0) G1(g2) G2(g1) ... G2(last): every down-GEMM tile comes after all
+// gate/up tiles of its group and of one more group, so by the time it is claimed the tiles
+// it depends on were claimed long before.
+__device__ __forceinline__ int build_tile_list(int4* tile_list, PlanState* plan, const int* cnt, const int* off, int E,
+                                                int NT1, int NT2, int T, int work_rows, int x_moe, int planned,
+                                                int n_extra_gemm) {
+  __shared__ ListScratch ls;
+  const int e = threadIdx.x;
+  const int we = (e < E) ? (cnt[e] + work_rows - 1) / work_rows : 0;
+  if (e < kMaxExperts) ls.work[e] = we;
+  int n_work;
+  const int w0 = block_excl_scan(we, &n_work, ls.warp_sums);
+  if (e < E) ls.w0[e] = w0;
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int ng = 0, acc = 0;
+    for (int x = 0; x < E; ++x) {
+      const int m = ls.work[x];
+      ls.grp[x] = ng;
+      ls.moff[x] = acc;
+      acc += m;
+      if (acc >= kGroupWork || x == E - 1) {
+        if (acc > 0) { ls.g_cnt[ng] = acc; ++ng; }
+        acc = 0;
+      }
+    }
+    int pos = 0;
+    for (int gi = 0; gi < ng; ++gi) {
+      ls.g_base1[gi] = pos;
+      pos += ls.g_cnt[gi] * NT1;
+      if (gi >= 1) { ls.g_base2[gi - 1] = pos; pos += ls.g_cnt[gi - 1] * NT2; }
+    }
+    if (ng > 0) { ls.g_base2[ng - 1] = pos; pos += ls.g_cnt[ng - 1] * NT2; }
+    ls.ntiles = pos;
+  }
+  __syncthreads();
+
+  // Inside an expert: n-major over its work tiles, so an expert's entries of one GEMM are one
+  // contiguous run of the list.  One warp per expert writes them (a popular expert has hundreds).
+  for (int x = threadIdx.x >> 5; x < E; x += 32) {
+    const int wx = ls.work[x];
+    if (wx == 0) continue;
+    const int lane = threadIdx.x & 31;
+    const int gi = ls.grp[x], cx = cnt[x], ox = off[x], mx = ls.w0[x];
+    const int b1 = ls.g_base1[gi] + ls.moff[x] * NT1, b2 = ls.g_base2[gi] + ls.moff[x] * NT2;
+    for (int i = lane; i < wx * NT1; i += 32) {
+      const int n = i / wx, j = i - n * wx;
+      tile_list[b1 + i] = make_entry(kGateUp, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
+    }
+    for (int i = lane; i < wx * NT2; i += 32) {
+      const int n = i / wx, j = i - n * wx;
+      tile_list[b2 + i] = make_entry(kDown, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
+    }
+  }
+  const int n_gemm = ls.ntiles;
+  const int n_comb = (T + kCombineTokens - 1) / kCombineTokens;
+  for (int c = threadIdx.x; c < n_comb; c += blockDim.x)
+    tile_list[n_gemm + c] = make_entry(kCombine, 0, c, c * kCombineTokens, min(kCombineTokens, T - c * kCombineTokens), 0);
+  if (threadIdx.x == 0) {
+    PlanState ps;
+    ps.n_mtiles = x_moe;
+    ps.n_gemm_tiles = n_gemm;
+    ps.n_comb_tiles = n_comb;
+    ps.planned = planned;                   // a plan with a rejected id leaves the slot without tiles to run
+    ps.n_extra_gemm = n_extra_gemm;
+    ps.pad[0] = ps.pad[1] = ps.pad[2] = 0;
+    *plan = ps;
+  }
+  __syncthreads();
+  return n_gemm;
+}
+
 // ---------------------------------------------------------------- K2: scans + tile table + tile list
 // the whole block of 1024 threads
 __device__ __forceinline__ void scan_body(const OpDev* __restrict__ op, int n_chunks, int R, int E, int NT1, int NT2,
                                           int T, int work_rows) {
   __shared__ int warp_sums[33];
-  __shared__ int s_cnt[kMaxExperts], s_grp[kMaxExperts], s_moff[kMaxExperts], s_off[kMaxExperts];
+  __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts];
   __shared__ int s_part[1024];
-  __shared__ int s_w0[kMaxExperts];
-  __shared__ int g_cnt[kMaxExperts], g_base1[kMaxExperts], g_base2[kMaxExperts];
-  __shared__ int s_ntiles;
   const int e = threadIdx.x;
 
   // column sums of the per-warp histograms, the device prefix sum over experts, then the base
@@ -153,70 +236,7 @@ __device__ __forceinline__ void scan_body(const OpDev* __restrict__ op, int n_ch
   }
   __syncthreads();
 
-  // Work tiles (the unit the queues hand out): up to `work_rows` consecutive rows of one
-  // expert, i.e. one or two adjacent m-tiles that share each weight tile they read.
-  // Dependency groups: consecutive experts holding at least kGroupWork work tiles.  The list
-  // is  G1(g0) G1(g1) G2(g0) G1(g2) G2(g1) ... G2(last): every down-GEMM tile comes after all
-  // gate/up tiles of its group and of one more group, so by the time it is claimed the tiles
-  // it depends on were claimed long before.
-  const int we = (e < E) ? (cnt + work_rows - 1) / work_rows : 0;
-  s_part[e] = we;                 // the column sums are consumed: the array now holds work tiles per expert
-  int n_work;
-  const int w0 = block_excl_scan(we, &n_work, warp_sums);
-  if (e < E) s_w0[e] = w0;
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int ng = 0, acc = 0;
-    for (int x = 0; x < E; ++x) {
-      const int m = s_part[x];
-      s_grp[x] = ng;
-      s_moff[x] = acc;
-      acc += m;
-      if (acc >= kGroupWork || x == E - 1) {
-        if (acc > 0) { g_cnt[ng] = acc; ++ng; }
-        acc = 0;
-      }
-    }
-    int pos = 0;
-    for (int gi = 0; gi < ng; ++gi) {
-      g_base1[gi] = pos;
-      pos += g_cnt[gi] * NT1;
-      if (gi >= 1) { g_base2[gi - 1] = pos; pos += g_cnt[gi - 1] * NT2; }
-    }
-    if (ng > 0) { g_base2[ng - 1] = pos; pos += g_cnt[ng - 1] * NT2; }
-    s_ntiles = pos;
-  }
-  __syncthreads();
-
-  // Inside an expert: n-major over its work tiles, so an expert's entries of one GEMM are one
-  // contiguous run of the list.  One warp per expert writes them (a popular expert has hundreds).
-  for (int x = threadIdx.x >> 5; x < E; x += 32) {
-    const int wx = s_part[x];
-    if (wx == 0) continue;
-    const int lane = threadIdx.x & 31;
-    const int gi = s_grp[x], cx = s_cnt[x], ox = s_off[x], mx = s_w0[x];
-    const int b1 = g_base1[gi] + s_moff[x] * NT1, b2 = g_base2[gi] + s_moff[x] * NT2;
-    for (int i = lane; i < wx * NT1; i += 32) {
-      const int n = i / wx, j = i - n * wx;
-      op->tile_list[b1 + i] = make_entry(kGateUp, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
-    }
-    for (int i = lane; i < wx * NT2; i += 32) {
-      const int n = i / wx, j = i - n * wx;
-      op->tile_list[b2 + i] = make_entry(kDown, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
-    }
-  }
-  const int n_gemm = s_ntiles;
-  const int n_comb = (T + kCombineTokens - 1) / kCombineTokens;
-  for (int c = threadIdx.x; c < n_comb; c += blockDim.x)
-    op->tile_list[n_gemm + c] = make_entry(kCombine, 0, c, c * kCombineTokens, min(kCombineTokens, T - c * kCombineTokens), 0);
-  if (threadIdx.x == 0) {
-    PlanState ps;
-    ps.n_mtiles = x_moe;
-    ps.n_gemm_tiles = n_gemm;
-    ps.n_comb_tiles = n_comb;
-    ps.planned = total == R ? 1 : 0;        // a plan with a rejected id leaves the slot without tiles to run
-    *op->plan = ps;
-  }
+  build_tile_list(op->tile_list, op->plan, s_cnt, s_off, E, NT1, NT2, T, work_rows, x_moe, total == R ? 1 : 0, 0);
 }
 
 __global__ void __launch_bounds__(1024)
@@ -289,6 +309,76 @@ plan_small_kernel(const OpDev* __restrict__ op, Global* g, int slot, int n_chunk
   __threadfence_block();
   __syncthreads();
   if (warp < n_chunks) scatter_chunk(op, R, E, warp, sm + warp * E, lane);
+}
+
+// ---------------------------------------------------------------- the paired form of a decode + prefill op
+// Two ops of one launch that share their expert weights can share weight tiles too.  The paired form puts
+// the routed rows of both into ONE packed row space -- per expert the prefill rows (in their plan's order)
+// followed by the decode rows (in theirs) -- and cuts it into two queue lists: per expert, the decode list
+// takes the decode rows plus as many of the prefill rows just before them as fit into the decode rows' last
+// tile of `carrier_rows` rows ("carrier" tiles: claimed with decode priority, they stream a weight tile once
+// for rows of both ops); the prefill list takes the rest.  Nothing about a row's arithmetic depends on the
+// tile it sits in, so the outputs are those of the unpaired ops, bit for bit.
+//   dp / pp: the paired descriptors (their PlanStates and lists are written here), d / p: the plain ones,
+//   whose counts and offsets the two moe_plan calls have written earlier on the stream.
+__global__ void __launch_bounds__(1024)
+plan_pair_kernel(const OpDev* dp, const OpDev* pp, const OpDev* d, const OpDev* p, int E, int NT1, int NT2,
+                 int work_rows, int carrier_rows) {
+  __shared__ int cnt_d[kMaxExperts], off_d[kMaxExperts], cnt_p[kMaxExperts], off_p[kMaxExperts];
+  const int e = threadIdx.x;
+  if (e < E) {
+    const int cd = d->counts[e], cp = p->counts[e];
+    const int moff = d->offsets[e] + p->offsets[e];
+    const int room = cd > 0 ? (cd + carrier_rows - 1) / carrier_rows * carrier_rows - cd : 0;
+    const int take = min(cp, room);
+    cnt_p[e] = cp - take;
+    off_p[e] = moff;
+    cnt_d[e] = cd + take;
+    off_d[e] = moff + cp - take;
+  }
+  __syncthreads();
+  const int ok = (d->plan->planned && p->plan->planned) ? 1 : 0;
+  const int n_dec = build_tile_list(dp->tile_list, dp->plan, cnt_d, off_d, E, NT1, NT2, d->n_tokens, carrier_rows,
+                                    d->plan->n_mtiles, ok, 0);
+  // every GEMM entry of the decode list may carry prefill rows: the prefill op is complete when they are too
+  build_tile_list(pp->tile_list, pp->plan, cnt_p, off_p, E, NT1, NT2, p->n_tokens, work_rows, p->plan->n_mtiles, ok,
+                  n_dec);
+}
+
+// the shared row space's permutation: for each op, flat routed index -> packed row, and packed row -> flat
+// index tagged with the slot the row belongs to
+__global__ void __launch_bounds__(256)
+plan_pair_scatter_kernel(const OpDev* d, const OpDev* p, int* gather_m, int* comb_d, int* comb_p, int Rd, int Rp, int E,
+                         int slot_d, int slot_p) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < Rd) {
+    const int e = d->topk_ids[i], ps = d->flat_to_sorted[i];
+    int m = -1;
+    if (e >= 0 && e < E && ps >= 0) {
+      m = ps + p->offsets[e + 1];               // behind the expert's prefill rows
+      gather_m[m] = i | (slot_d << kRowSlotShift);
+    }
+    comb_d[i] = m;
+  } else if (i < Rd + Rp) {
+    const int j = i - Rd;
+    const int e = p->topk_ids[j], ps = p->flat_to_sorted[j];
+    int m = -1;
+    if (e >= 0 && e < E && ps >= 0) {
+      m = ps + d->offsets[e];                   // shifted by the decode rows of the experts before
+      gather_m[m] = j | (slot_p << kRowSlotShift);
+    }
+    comb_p[j] = m;
+  }
+}
+
+cudaError_t launch_plan_pair(const OpDev* dp, const OpDev* pp, const OpDev* d, const OpDev* p, int* gather_m, int* comb_d,
+                             int* comb_p, int Rd, int Rp, int E, int NT1, int NT2, int work_rows, int carrier_rows,
+                             int slot_d, int slot_p, cudaStream_t stream) {
+  plan_pair_kernel<<<1, 1024, 0, stream>>>(dp, pp, d, p, E, NT1, NT2, work_rows, carrier_rows);
+  const int n = Rd + Rp;
+  if (n > 0)
+    plan_pair_scatter_kernel<<<(n + 255) / 256, 256, 0, stream>>>(d, p, gather_m, comb_d, comb_p, Rd, Rp, E, slot_d, slot_p);
+  return cudaGetLastError();
 }
 
 cudaError_t prepare_plan_kernels() {

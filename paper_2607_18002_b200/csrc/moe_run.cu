@@ -32,6 +32,7 @@
 #include "moe_ptx.cuh"
 #include "moe_sched.cuh"
 #include <cuda_fp8.h>
+#include <climits>
 
 namespace moe {
 
@@ -84,13 +85,18 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
   const float* sx;
   const float *sw0, *sw1;
   if (g1) {
+    // the row's activation scales: its own op's, or (paired form) the partner's when the row is tagged so
     int tok = 0;
+    const OpDev* src = op;
     if (valid) {
-      const int flat = op->sorted_to_flat[ti.row0 + row];
-      if ((unsigned)flat < (unsigned)op->n_rows) tok = flat / a.k;
-      else report(c.st, MOE_EBOUNDS, ti.slot, ti.row0 + row, flat, 1);
+      const int v = op->gather_list[ti.row0 + row];
+      const int tag = v >> kRowSlotShift, flat = v & kRowFlatMask;
+      const int own_tag = op->paired ? slot_of(&a, ti.slot) : 0;
+      if (op->paired && tag != own_tag && tag == slot_of(&a, op->partner)) src = &a.ops[op->partner];
+      if (v >= 0 && (tag == own_tag || src != op) && flat < src->n_rows) tok = flat / a.k;
+      else { src = op; report(c.st, MOE_EBOUNDS, slot_of(&a, ti.slot), ti.row0 + row, v, 1); }
     }
-    sx = op->x_scale + (size_t)tok * HB;
+    sx = src->x_scale + (size_t)tok * HB;
     sw0 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + ti.n) * HB;
     sw1 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + IB + ti.n) * HB;
   } else {
@@ -294,7 +300,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         if (lane == 0) {
           // a claimed tile only ever waits on tiles that were claimed before it
           if (ti.kind == kDown) ok = wait_counter(c, &op->g1_done[ti.m], args.I / kTileN1, 3);
-          if (ti.kind == kCombine) ok = wait_counter(c, &op->run->gemm_done, op->plan->n_gemm_tiles, 4);
+          if (ti.kind == kCombine) ok = wait_counter(c, &op->run->gemm_done, op_gemm_tiles(op), 4);
           if (!ok) ti.kind = kEnd;
           fence_async_proxy();
           sc->info[islot] = ti;
@@ -340,7 +346,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
               int met = 1;
               if (lane == 0) {
                 if (nx.kind == kDown) met = ld_acquire(&nop->g1_done[nx.m]) >= args.I / kTileN1;
-                if (nx.kind == kCombine) met = ld_acquire(&nop->run->gemm_done) >= nop->plan->n_gemm_tiles;
+                if (nx.kind == kCombine) met = ld_acquire(&nop->run->gemm_done) >= op_gemm_tiles(nop);
                 if (met) {
                   fence_async_proxy();
                   sc->info[islot] = nx;
@@ -496,33 +502,45 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         continue;
       }
       const OpDev* op = &args.ops[slot];
+      // a paired op's gather list also holds rows of its partner, tagged with their slot: those come from
+      // the partner's activations (kept as the complement of the token index)
+      const bool paired = op->paired != 0;
+      const OpDev* pop = paired ? &args.ops[op->partner] : op;
       const unsigned char* X = static_cast<const unsigned char*>(op->x) + chunk * 16;
+      const unsigned char* Xp = static_cast<const unsigned char*>(pop->x) + chunk * 16;
       const size_t pitch = (size_t)args.H * kEl;
       int tok[kPasses];
-      const int n_rows = op->n_rows;
+      const int n_rows = op->n_rows, n_rows_p = pop->n_rows;
+      const int own_tag = paired ? slot_of(&args, slot) : 0, partner_tag = paired ? slot_of(&args, op->partner) : 0;
       bool bad = false;
 #pragma unroll
       for (int j = 0; j < kPasses; ++j) {
         const int r = rbase + kRowsPerPass * j;
-        const int flat = r < rows ? op->sorted_to_flat[row0 + r] : 0;
-        const bool in_range = (unsigned)flat < (unsigned)n_rows;    // an index the plan never wrote is reported
-        bad |= !in_range;                                            // below and its row is skipped
-        tok[j] = (r < rows && in_range) ? flat / args.k : -1;
+        const int v = r < rows ? op->gather_list[row0 + r] : 0;
+        const int tag = v >> kRowSlotShift, flat = v & kRowFlatMask;
+        const bool theirs = tag != own_tag;
+        // an index the plan never wrote is reported below and its row is skipped
+        const bool in_range = v >= 0 && (tag == own_tag || tag == partner_tag) && flat < (theirs ? n_rows_p : n_rows);
+        bad |= !in_range;
+        tok[j] = (r < rows && in_range) ? (theirs ? ~(flat / args.k) : flat / args.k) : INT_MIN;
       }
-      if (bad) report(c.st, MOE_EBOUNDS, slot, row0, rows, 0);
+      if (bad) report(c.st, MOE_EBOUNDS, slot_of(&args, slot), row0, rows, 0);
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
         const int stage = (int)(kiter % kNS);
         if (!__all_sync(0xffffffffu, mbar_wait(c, &sc->empty[stage], ((kiter / kNS) & 1u) ^ 1u, 14))) { fail = true; break; }
         const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
         const unsigned char* Xk = X + (size_t)kb * kRowBytes;
+        const unsigned char* Xpk = Xp + (size_t)kb * kRowBytes;
 #pragma unroll
         for (int j = 0; j < kPasses; ++j) {
           const int r = rbase + kRowsPerPass * j;
           // the swizzle XORs the 16-byte chunk index with the row's position in its 8-row group
           const int sw = kRowBytes == 128 ? (r & 7) : ((r >> 1) & 3);
-          if (tok[j] >= 0)
-            cp_async_16(sA + r * kRowBytes + ((chunk ^ sw) << 4), Xk + (size_t)tok[j] * pitch);
+          const int t = tok[j];
+          if (t != INT_MIN)
+            cp_async_16(sA + r * kRowBytes + ((chunk ^ sw) << 4),
+                        (t >= 0 ? Xk : Xpk) + (size_t)(t >= 0 ? t : ~t) * pitch);
         }
         cp_async_arrive_noinc(&sc->fullA[stage]);
       }

@@ -22,6 +22,7 @@
 #include "moe_combine.cuh"
 #include "moe_ptx.cuh"
 #include "moe_sched.cuh"
+#include <climits>
 
 namespace moe {
 namespace pairk {
@@ -272,7 +273,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       int ok = 1;
       if (lane == 0) {
         if (ti.kind == kDown) ok = wait_counter(c, &op->g1_done[ti.m], args.I / kTileN1, 3);
-        if (ti.kind == kCombine) ok = wait_counter(c, &op->run->gemm_done, op->plan->n_gemm_tiles, 4);
+        if (ti.kind == kCombine) ok = wait_counter(c, &op->run->gemm_done, op_gemm_tiles(op), 4);
         if (!ok) ti.kind = kEnd;
         publish(sc, islot, ti);
       }
@@ -280,7 +281,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       ti.kind = __shfl_sync(0xffffffffu, ti.kind, 0);
       // The gather warps will read the tile's row list (4 bytes per row) first thing: pull it into L2
       // now, the weight stream has usually pushed it out since the plan wrote it.
-      if (ti.kind == kGateUp && lane * 32 < ti.rows) prefetch_l2(op->sorted_to_flat + ti.row0 + lane * 32);
+      if (ti.kind == kGateUp && lane * 32 < ti.rows) prefetch_l2(op->gather_list + ti.row0 + lane * 32);
       if (ti.kind == kEnd || !ok) break;
       if (!wwait(c, &sc->taken[islot], iph, 26)) break;
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
@@ -422,22 +423,32 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
       if (kind == kCombine) continue;
       if (kind != kGateUp) { kiter += (unsigned)kblocks; continue; }
       const OpDev* op = &args.ops[slot];
+      // a paired op's gather list also holds rows of its partner, tagged with their slot: those come from
+      // the partner's activations (kept as the complement of the token index)
+      const bool paired = op->paired != 0;
+      const OpDev* pop = paired ? &args.ops[op->partner] : op;
       const unsigned char* X = static_cast<const unsigned char*>(op->x) + chunk * 16;
+      const unsigned char* Xp = static_cast<const unsigned char*>(pop->x) + chunk * 16;
       const size_t pitch = (size_t)args.H * 2;
       const int rpc = rows > kTileM ? 128 : 64;
       const int first = rank * rpc;                       // this CTA's first row of the tile
       int tok[kPasses];
-      const int n_rows = op->n_rows;
+      const int n_rows = op->n_rows, n_rows_p = pop->n_rows;
+      const int own_tag = paired ? slot_of(&args, slot) : 0, partner_tag = paired ? slot_of(&args, op->partner) : 0;
       bool bad = false;
 #pragma unroll
       for (int j = 0; j < kPasses; ++j) {
         const int r = rbase + kRowsPerPass * j;
-        const int flat = (r < rpc && first + r < rows) ? op->sorted_to_flat[row0 + first + r] : 0;
-        const bool in_range = (unsigned)flat < (unsigned)n_rows;    // an index the plan never wrote is reported
-        bad |= !in_range;                                            // below and its row is skipped
-        tok[j] = (r < rpc && first + r < rows && in_range) ? flat / args.k : -1;
+        const bool mine = r < rpc && first + r < rows;
+        const int v = mine ? op->gather_list[row0 + first + r] : 0;
+        const int tag = v >> kRowSlotShift, flat = v & kRowFlatMask;
+        const bool theirs = tag != own_tag;
+        // an index the plan never wrote is reported below and its row is skipped
+        const bool in_range = v >= 0 && (tag == own_tag || tag == partner_tag) && flat < (theirs ? n_rows_p : n_rows);
+        bad |= !in_range;
+        tok[j] = (mine && in_range) ? (theirs ? ~(flat / args.k) : flat / args.k) : INT_MIN;
       }
-      if (bad) report(c.st, MOE_EBOUNDS, slot, row0, rows, 0);
+      if (bad) report(c.st, MOE_EBOUNDS, slot_of(&args, slot), row0, rows, 0);
       unsigned long long* landed = leader ? sc->full : sc->fullA;
       bool fail = false;
       for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
@@ -446,11 +457,14 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
         gmask ^= 1u << stage;
         const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
         const unsigned char* Xk = X + (size_t)kb * kRowBytes;
+        const unsigned char* Xpk = Xp + (size_t)kb * kRowBytes;
 #pragma unroll
         for (int j = 0; j < kPasses; ++j) {
           const int r = rbase + kRowsPerPass * j;
-          if (tok[j] >= 0)     // the swizzle XORs the chunk index with the row's place in its 8-row group
-            cp_async_16(sA + r * kRowBytes + ((chunk ^ (r & 7)) << 4), Xk + (size_t)tok[j] * pitch);
+          const int t = tok[j];
+          if (t != INT_MIN)    // the swizzle XORs the chunk index with the row's place in its 8-row group
+            cp_async_16(sA + r * kRowBytes + ((chunk ^ (r & 7)) << 4),
+                        (t >= 0 ? Xk : Xpk) + (size_t)(t >= 0 ? t : ~t) * pitch);
         }
         cp_async_arrive_noinc(&landed[stage]);
       }

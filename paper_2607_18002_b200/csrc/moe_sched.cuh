@@ -97,14 +97,21 @@ __device__ __noinline__ inline bool wait_counter(const Ctx& c, const int* p, int
 // a slot whose plan was rejected (an expert id out of range) holds no tiles
 __device__ __forceinline__ int op_total_tiles(const OpDev* op, int fuse) {
   if (op->plan->planned == 0) return 0;
+  return op->plan->n_gemm_tiles + op->plan->n_extra_gemm + (fuse ? op->plan->n_comb_tiles : 0);
+}
+// entries of the op's own queue list
+__device__ __forceinline__ int op_queue_entries(const OpDev* op, int fuse) {
+  if (op->plan->planned == 0) return 0;
   return op->plan->n_gemm_tiles + (fuse ? op->plan->n_comb_tiles : 0);
 }
+// GEMM entries that must have committed before the op's combine may run
+__device__ __forceinline__ int op_gemm_tiles(const OpDev* op) { return op->plan->n_gemm_tiles + op->plan->n_extra_gemm; }
 
 // An op without tiles (no tokens, or a plan that was rejected) never commits anything: it counts as
 // finished as soon as its own predecessor has, and its ready word is not consulted.
 __device__ inline bool op_finished(const RunArgs* a, int slot) {
   for (int hop = 0; slot >= 0 && hop <= kMaxOps; ++hop) {
-    const OpDev* op = &a->ops[slot];
+    const OpDev* op = &a->ops[a->desc[slot]];
     if (op_total_tiles(op, a->fuse_combine) > 0) return ld_acquire(&op->run->done) != 0;
     slot = op->after_op;
   }
@@ -124,7 +131,7 @@ __device__ inline void finish_empty_ops(const RunArgs* a, int finished) {
     OpDev* op = &a->ops[a->slots[i]];
     if (op_total_tiles(op, a->fuse_combine) > 0) continue;
     int dep = op->after_op;
-    for (int hop = 0; dep >= 0 && hop <= kMaxOps && op_total_tiles(&a->ops[dep], a->fuse_combine) == 0; ++hop)
+    for (int hop = 0; dep >= 0 && hop <= kMaxOps && op_total_tiles(&a->ops[a->desc[dep]], a->fuse_combine) == 0; ++hop)
       dep = a->ops[dep].after_op;
     if (dep != finished) continue;
     atomicExch(&op->run->done, 1);
@@ -151,8 +158,12 @@ __device__ inline int try_claim(const RunArgs* a, QueueTables* sc, RunHead* rh, 
   int slot = sc->cls_slot[cls][i];
   const OpDev* op = &a->ops[slot];
   if (!sc->cls_free[cls][i] && !op_ready(a, op)) return -1;
-  // the 32 entries from the head on are fetched while the fetch-add is in flight
   const unsigned base = h - sc->cum[cls][i];
+  // The head stands at the op's combine entries while GEMM entries they depend on are still running
+  // (other units hold them; for a paired prefill op, the decode list's carrier tiles): nothing to take here
+  // yet -- the caller turns to the other class instead of holding a combine ticket it cannot run.
+  if (base >= (unsigned)op->plan->n_gemm_tiles && ld_acquire(&op->run->gemm_done) < op_gemm_tiles(op)) return -1;
+  // the 32 entries from the head on are fetched while the fetch-add is in flight
   const unsigned n_op = sc->cum[cls][i + 1] - sc->cum[cls][i];
   int4 e = make_int4(0, 0, 0, 0);
   if (base + lane < n_op) e = op->tile_list[base + lane];
@@ -225,7 +236,7 @@ __device__ inline bool wait_op_ready(const Ctx& c, int lane, const TileInfo& ti)
     __nanosleep(256);
     if (aborted(c)) return false;
     if ((long long)(gtime_ns() - w0) > a->wait_ns) {
-      if (lane == 0) report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, ti.slot, ti.tile);
+      if (lane == 0) report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, slot_of(a, ti.slot), ti.tile);
       return false;
     }
   }
@@ -276,6 +287,19 @@ __device__ inline void claim_next(const Ctx& c, QueueTables* sc, RunHead* rh, in
   ti.kind = kEnd;
 }
 
+// one committed entry counted for `op` (descriptor `desc`): counters, notify word, completion
+__device__ inline void count_commit(const RunArgs* a, OpDev* op, int desc, bool gemm) {
+  if (gemm) atomicAdd(&op->run->gemm_done, 1);
+  const int done = atomicAdd(&op->run->tiles_done, 1) + 1;
+  if (op->notify != nullptr && done == op->notify_after) st_release_sys(op->notify, 1u);
+  if (done == op_total_tiles(op, a->fuse_combine)) {
+    __threadfence();
+    atomicExch(&op->run->done, 1);
+    if (op->done != nullptr) st_release_sys(op->done, 1u);
+    finish_empty_ops(a, slot_of(a, desc));
+  }
+}
+
 // Publishing a finished tile: dependency counter, op completion, done word, log.
 // Called by one thread after all writers of the tile have fenced and synchronised.
 __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti) {
@@ -285,22 +309,16 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
   fence_async_proxy();
   const unsigned long long t_commit = a->log_cap > 0 ? gtime_ns() : 0ull;   // before it is published
   if (ti.kind == kGateUp) atomicAdd(&op->g1_done[ti.m], 1);
-  if (ti.kind != kCombine) atomicAdd(&op->run->gemm_done, 1);
-  const int done = atomicAdd(&op->run->tiles_done, 1) + 1;
-  if (op->notify != nullptr && done == op->notify_after) st_release_sys(op->notify, 1u);
-  if (done == op_total_tiles(op, a->fuse_combine)) {
-    __threadfence();
-    atomicExch(&op->run->done, 1);
-    if (op->done != nullptr) st_release_sys(op->done, 1u);
-    finish_empty_ops(a, ti.slot);
-  }
+  count_commit(a, op, ti.slot, ti.kind != kCombine);
+  // a GEMM entry of a paired decode op carries rows of the prefill op too: it counts for both
+  if (op->paired && op->cls == MOE_CLASS_DECODE && ti.kind != kCombine) count_commit(a, &a->ops[op->partner], op->partner, true);
   if (a->log_cap > 0) {
     const unsigned idx = atomicAdd(&rh->log_count, 1u);
     if (idx < (unsigned)a->log_cap) {
       moe_tile_rec_t r;
       r.t_claim = ti.t_claim;
       r.t_commit = t_commit;
-      r.slot = ti.slot;
+      r.slot = slot_of(a, ti.slot);
       r.tile = ti.tile;
       r.cls = (int16_t)ti.cls;
       r.kind = (int16_t)ti.kind;
@@ -323,7 +341,7 @@ __device__ inline void build_queues(const RunArgs* a, QueueTables* sc) {
     const int j = sc->n_cls[cls]++;
     sc->cls_slot[cls][j] = slot;
     sc->cls_free[cls][j] = (op->ready == nullptr && op->after_op < 0) ? 1 : 0;
-    sc->cum[cls][j + 1] = sc->cum[cls][j] + (unsigned)op_total_tiles(op, a->fuse_combine);
+    sc->cum[cls][j + 1] = sc->cum[cls][j] + (unsigned)op_queue_entries(op, a->fuse_combine);
   }
 }
 
