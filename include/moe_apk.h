@@ -48,6 +48,12 @@ enum {
 
 enum { MOE_DTYPE_BF16 = 0, MOE_DTYPE_FP8_E4M3 = 1 };
 enum { MOE_CLASS_DECODE = 0, MOE_CLASS_PREFILL = 1 };
+/* How an op's activations are laid out (Section 2.4).  GATHERED: x is [T, H] in token order and the
+ * plan packs the routed rows per expert (the contiguous layout).  MASKED: x already sits in per-expert
+ * slabs [E, slab_rows, H] of which the first counts[e] rows of slab e are valid (what a dispatch step
+ * of fixed-size buffers delivers, and what decode under captured graphs uses): nothing is permuted,
+ * y is written in the same slab layout and there is no combine. */
+enum { MOE_LAYOUT_GATHERED = 0, MOE_LAYOUT_MASKED = 1 };
 
 /* Height of a token-dimension tile (the M_t of the footprint formula, Section 6.2). */
 #define MOE_TILE_M 128
@@ -94,6 +100,11 @@ typedef struct {
   int32_t decode_sms;     /* the SM budget field of the op template (Section 4.2): > 0    */
                           /* makes the decode budget take this value when the op's first  */
                           /* tile is claimed, 0 leaves the budget word alone              */
+  int32_t layout;         /* MOE_LAYOUT_*.  MASKED: n_tokens is ignored; x and y are       */
+  int32_t slab_rows;      /* [E, slab_rows, H] (x_scale [E, slab_rows, H/128]); counts [E] */
+                          /* is an INPUT (valid rows per slab, 0..slab_rows); offsets is   */
+                          /* still written; topk_ids, topk_w and the permutations are not  */
+                          /* used; E * slab_rows <= max_tokens_per_op * top_k              */
 } moe_op_t;
 
 /* One record per executed tile (only when tile_log_entries > 0). Times are GPU
@@ -104,7 +115,8 @@ typedef struct {
   uint64_t t_commit; /* its outputs are written and published                             */
   int32_t slot;      /* op slot                                                           */
   int32_t tile;      /* index in the op's tile list                                       */
-  int16_t cls, kind; /* class; 0 = gate/up GEMM + SwiGLU, 1 = down GEMM, 2 = combine      */
+  int16_t cls, kind; /* class; 0 = gate/up GEMM + SwiGLU, 1 = down GEMM, 2 = combine,     */
+                     /* 3 = gate/up GEMM + SwiGLU of a masked-layout op                   */
   int16_t cta, sm;   /* CTA index and SM id that ran it (first CTA of a pair)                */
 } moe_tile_rec_t;
 

@@ -24,6 +24,7 @@ MOE_OK, MOE_EINVAL, MOE_ENOSPC, MOE_ECUDA = 0, -1, -2, -3
 MOE_ETIMEOUT, MOE_EBADID, MOE_EBOUNDS, MOE_ENOTPLANNED = -4, -5, -6, -7
 MOE_DTYPE_BF16, MOE_DTYPE_FP8_E4M3 = 0, 1
 MOE_CLASS_DECODE, MOE_CLASS_PREFILL = 0, 1
+MOE_LAYOUT_GATHERED, MOE_LAYOUT_MASKED = 0, 1
 MOE_TILE_M = 128
 
 EXPORTS = ("moe_workspace_bytes", "moe_create", "moe_destroy", "moe_plan", "moe_run",
@@ -56,7 +57,7 @@ class moe_op_t(C.Structure):
                 ("sorted_to_flat", C.c_void_p), ("flat_to_sorted", C.c_void_p),
                 ("ready", C.c_void_p), ("done", C.c_void_p),
                 ("after_op", C.c_int32), ("notify_after", C.c_int32), ("notify", C.c_void_p),
-                ("decode_sms", C.c_int32)]
+                ("decode_sms", C.c_int32), ("layout", C.c_int32), ("slab_rows", C.c_int32)]
 
 
 class moe_tile_rec_t(C.Structure):
@@ -285,7 +286,24 @@ def bind_op(cls: int, x, topk_ids, topk_w, w_gate_up, w_down, top_k: int, n_expe
     c_op = moe_op_t(cls, T, _ptr(x), _ptr(x_scale), _ptr(topk_ids), _ptr(topk_w),
                     _ptr(w_gate_up), _ptr(w_down), _ptr(s_gate_up), _ptr(s_down), _ptr(y),
                     _ptr(counts), _ptr(offsets), _ptr(s2f), _ptr(f2s), _ptr(ready), _ptr(done),
-                    after_op, notify_after, _ptr(notify), decode_sms)
+                    after_op, notify_after, _ptr(notify), decode_sms, MOE_LAYOUT_GATHERED, 0)
+    return BoundOp(c_op, keep)
+
+
+def bind_masked_op(cls: int, x_slabs, counts, w_gate_up, w_down, x_scale=None, s_gate_up=None, s_down=None,
+                   ready=None, done=None, after_op: int = -1, decode_sms: int = 0) -> BoundOp:
+    """A masked-layout op: x_slabs [E, slab_rows, H] (its scales [E, slab_rows, H/128] for e4m3), counts int32 [E]
+    valid rows per slab.  Allocates y in the same slab layout and the offsets output."""
+    import torch
+    E, slab_rows, H = (int(v) for v in x_slabs.shape)
+    dev = w_gate_up.device
+    y = torch.zeros((E, slab_rows, H), dtype=torch.bfloat16, device=dev)
+    offsets = torch.empty(E + 1, dtype=torch.int32, device=dev)
+    keep = dict(x=x_slabs, x_scale=x_scale, w_gate_up=w_gate_up, w_down=w_down, s_gate_up=s_gate_up, s_down=s_down,
+                y=y, counts=counts, offsets=offsets, ready=ready, done=done)
+    c_op = moe_op_t(cls, 0, _ptr(x_slabs), _ptr(x_scale), None, None, _ptr(w_gate_up), _ptr(w_down), _ptr(s_gate_up),
+                    _ptr(s_down), _ptr(y), _ptr(counts), _ptr(offsets), None, None, _ptr(ready), _ptr(done),
+                    after_op, 0, None, decode_sms, MOE_LAYOUT_MASKED, slab_rows)
     return BoundOp(c_op, keep)
 
 

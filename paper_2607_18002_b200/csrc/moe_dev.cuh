@@ -25,7 +25,9 @@ constexpr int kWorkRowsFp8 = 128;    // fp8: the accumulator and both partial bu
 constexpr int kMaxOps = 16;
 constexpr int kMaxExperts = 1024;
 
-enum TileKind : int { kGateUp = 0, kDown = 1, kCombine = 2 };
+// kGateUpDirect: a gate/up tile whose activation rows are consecutive rows of x (masked layout): they are
+// loaded by TMA like the rows of a down tile instead of being gathered through a permutation
+enum TileKind : int { kGateUp = 0, kDown = 1, kCombine = 2, kGateUpDirect = 3 };
 
 // Queue entry (16 bytes, one load per claim): x = kind | n-tile << 4 | m-tile << 12,
 // y = first packed row (first token for a combine tile), z = valid rows, w = expert.
@@ -68,6 +70,10 @@ struct __align__(128) OpDev {
   CUtensorMap tm_a128;  // [Rmax, I]   box {64, 128}
   CUtensorMap tm_a256;  // [Rmax, I]   box {64, 256}
   CUtensorMap tm_w1h;   // [E*2I, H]   box {64, 64}  gate/up weights, half-height box (CTA-pair kernel)
+  CUtensorMap tm_x8;    // masked layout only: x as [E*slab_rows, H], boxes of 8 / 32 / 128 / 256 rows
+  CUtensorMap tm_x32;
+  CUtensorMap tm_x128;
+  CUtensorMap tm_x256;
   int cls, n_tokens, n_rows, after_op;
   const void* x;
   const float* x_scale;
@@ -105,9 +111,10 @@ struct __align__(128) OpDev {
   const int* gather_list;   // packed row -> flat routed index (paired: | slot << kRowSlotShift)
   const int* comb_index;    // flat routed index -> packed row of D
   int space_rows;           // rows of the packed space that A, D and comb_index refer to
+  int masked;               // 1: masked layout (x, A, y in per-expert slabs of slab_rows rows)
   int paired;               // 1: this is the paired form of the slot
   int partner;              // paired: descriptor index of the other op of the pair, else -1
-  int pad_[3];
+  int pad_[2];
 };
 constexpr int kRowSlotShift = 27;                       // a flat routed index stays below 2^27 (moe_create checks)
 constexpr int kRowFlatMask = (1 << kRowSlotShift) - 1;

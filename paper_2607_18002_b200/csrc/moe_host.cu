@@ -11,6 +11,8 @@
 namespace moe {
 cudaError_t launch_plan(const OpDev* d_op, Global* g, int slot, int T, int k, int E, int NT1,
                         int NT2, int work_rows, cudaStream_t stream);
+cudaError_t launch_plan_masked(const OpDev* d_op, Global* g, int slot, int E, int NT1, int NT2, int slab_rows, int work_rows,
+                               cudaStream_t stream);
 cudaError_t launch_plan_pair(const OpDev* dp, const OpDev* pp, const OpDev* d, const OpDev* p, int* gather_m, int* comb_d,
                              int* comb_p, int Rd, int Rp, int E, int NT1, int NT2, int work_rows, int carrier_rows,
                              int slot_d, int slot_p, cudaStream_t stream);
@@ -240,16 +242,22 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   const moe_config_t& c = ctx->cfg;
   if (slot < 0 || slot >= c.max_ops) return MOE_EINVAL;
   if (op->cls != MOE_CLASS_DECODE && op->cls != MOE_CLASS_PREFILL) return MOE_EINVAL;
+  const bool masked = op->layout == MOE_LAYOUT_MASKED;
+  if (op->layout != MOE_LAYOUT_GATHERED && !masked) return MOE_EINVAL;
   if (op->n_tokens < 0) return MOE_EINVAL;
-  if (op->n_tokens > c.max_tokens_per_op) return MOE_ENOSPC;
+  if (!masked && op->n_tokens > c.max_tokens_per_op) return MOE_ENOSPC;
   if (op->after_op < -1 || op->after_op >= c.max_ops || op->after_op == slot) return MOE_EINVAL;
   if (op->notify && op->notify_after < 1) return MOE_EINVAL;
   if (op->decode_sms < 0) return MOE_EINVAL;
   if (!op->counts || !op->offsets) return MOE_EINVAL;
   if (!op->w_gate_up || !op->w_down || !aligned16(op->w_gate_up) || !aligned16(op->w_down)) return MOE_EINVAL;
-  if (c.dtype == MOE_DTYPE_FP8_E4M3 && (!op->s_gate_up || !op->s_down || (op->n_tokens > 0 && !op->x_scale)))
+  if (c.dtype == MOE_DTYPE_FP8_E4M3 && (!op->s_gate_up || !op->s_down || ((op->n_tokens > 0 || masked) && !op->x_scale)))
     return MOE_EINVAL;
-  if (op->n_tokens > 0) {
+  if (masked) {
+    if (op->slab_rows < 1 || !op->x || !op->y || !aligned16(op->x) || !aligned16(op->y)) return MOE_EINVAL;
+    // the slabs of the intermediate live in the slot's scratch, one row per slab row
+    if ((long long)c.n_experts * op->slab_rows > (long long)c.max_tokens_per_op * c.top_k) return MOE_ENOSPC;
+  } else if (op->n_tokens > 0) {
     if (!op->x || !op->topk_ids || !op->topk_w || !op->y || !op->sorted_to_flat || !op->flat_to_sorted)
       return MOE_EINVAL;
     if (!aligned16(op->x) || !aligned16(op->y)) return MOE_EINVAL;
@@ -259,8 +267,8 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   OpDev h;
   memset(&h, 0, sizeof(h));
   h.cls = op->cls;
-  h.n_tokens = op->n_tokens;
-  h.n_rows = op->n_tokens * c.top_k;
+  h.n_tokens = masked ? 0 : op->n_tokens;                     // a masked op has no token-order output to combine
+  h.n_rows = masked ? c.n_experts * op->slab_rows : op->n_tokens * c.top_k;
   h.after_op = op->after_op;
   h.x = op->x; h.x_scale = op->x_scale; h.topk_ids = op->topk_ids; h.topk_w = op->topk_w;
   h.w_gate_up = op->w_gate_up; h.w_down = op->w_down; h.s_gate_up = op->s_gate_up; h.s_down = op->s_down;
@@ -271,7 +279,9 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   h.op_budget = op->decode_sms;
   h.A = reinterpret_cast<__nv_bfloat16*>(sb + L.A_off);
   h.a_scale = reinterpret_cast<float*>(sb + L.A_off + align_up((size_t)L.max_rows * c.inter, 16));
-  h.D = reinterpret_cast<__nv_bfloat16*>(sb + L.D_off);
+  // masked layout: the expert outputs ARE the op's output, in the slab layout of x
+  h.D = masked ? static_cast<__nv_bfloat16*>(op->y) : reinterpret_cast<__nv_bfloat16*>(sb + L.D_off);
+  h.masked = masked ? 1 : 0;
   h.mtiles = reinterpret_cast<MTile*>(sb + L.mtiles_off);
   h.tile_list = reinterpret_cast<int4*>(sb + L.tiles_off);
   h.plan_hist = reinterpret_cast<int*>(sb + L.hist_off);
@@ -295,7 +305,7 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (!same) {
     int rc = MOE_OK;
-    if (op->n_tokens > 0) {
+    if (op->n_tokens > 0 || masked) {
       rc = make_map(ctx, &h.tm_a8, h.A, (size_t)L.max_rows, (size_t)c.inter, 8);
       if (!rc) rc = make_map(ctx, &h.tm_a32, h.A, (size_t)L.max_rows, (size_t)c.inter, 32);
       if (!rc) rc = make_map(ctx, &h.tm_a128, h.A, (size_t)L.max_rows, (size_t)c.inter, 128);
@@ -303,6 +313,13 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
       if (!rc) rc = make_map(ctx, &h.tm_w1, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 128);
       if (!rc) rc = make_map(ctx, &h.tm_w1h, op->w_gate_up, (size_t)c.n_experts * 2 * c.inter, (size_t)c.hidden, 64);
       if (!rc) rc = make_map(ctx, &h.tm_w2, op->w_down, (size_t)c.n_experts * c.hidden, (size_t)c.inter, 128);
+      if (masked) {
+        const size_t xr = (size_t)c.n_experts * op->slab_rows;
+        if (!rc) rc = make_map(ctx, &h.tm_x8, op->x, xr, (size_t)c.hidden, 8);
+        if (!rc) rc = make_map(ctx, &h.tm_x32, op->x, xr, (size_t)c.hidden, 32);
+        if (!rc) rc = make_map(ctx, &h.tm_x128, op->x, xr, (size_t)c.hidden, 128);
+        if (!rc) rc = make_map(ctx, &h.tm_x256, op->x, xr, (size_t)c.hidden, 256);
+      }
       if (rc) return rc;
     }
     ctx->planned[slot] = false;
@@ -312,8 +329,12 @@ int moe_plan(moe_ctx_t* ctx, int slot, const moe_op_t* op, void* stream) {
     ctx->ops[slot] = *op;             // what the device copy of the slot now describes
     ctx->uploaded[slot] = true;
   }
-  if (launch_plan(ctx->op_dev(slot), ctx->g(), slot, op->n_tokens, c.top_k, c.n_experts, L.NT1, L.NT2,
-                  c.dtype == MOE_DTYPE_FP8_E4M3 ? kWorkRowsFp8 : kWorkRowsBf16, st) != cudaSuccess) {
+  const int work_rows = c.dtype == MOE_DTYPE_FP8_E4M3 ? kWorkRowsFp8 : kWorkRowsBf16;
+  const cudaError_t pe = masked ? launch_plan_masked(ctx->op_dev(slot), ctx->g(), slot, c.n_experts, L.NT1, L.NT2,
+                                                     op->slab_rows, work_rows, st)
+                                : launch_plan(ctx->op_dev(slot), ctx->g(), slot, op->n_tokens, c.top_k, c.n_experts, L.NT1,
+                                              L.NT2, work_rows, st);
+  if (pe != cudaSuccess) {
     ctx->planned[slot] = false;
     return MOE_ECUDA;
   }
@@ -404,13 +425,16 @@ int moe_run_plain(moe_ctx_t* ctx, int slot, void* stream) {
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
   a.static_kind = 0;
   if (ps.n_gemm_tiles > 0 && launch_pair(a, ctx->rh(), 2 * ps.n_gemm_tiles, st) != cudaSuccess) return MOE_ECUDA;
-  if (launch_combine(ctx->op_dev(slot), ctx->ops[slot].n_tokens, c.top_k, c.hidden, st) != cudaSuccess) return MOE_ECUDA;
+  if (ctx->ops[slot].layout == MOE_LAYOUT_GATHERED &&
+      launch_combine(ctx->op_dev(slot), ctx->ops[slot].n_tokens, c.top_k, c.hidden, st) != cudaSuccess)
+    return MOE_ECUDA;
   return MOE_OK;
 }
 
 int moe_combine(moe_ctx_t* ctx, int slot, void* stream) {
   if (!ctx || slot < 0 || slot >= ctx->cfg.max_ops) return MOE_EINVAL;
   if (!ctx->planned[slot]) return MOE_ENOTPLANNED;
+  if (ctx->ops[slot].layout != MOE_LAYOUT_GATHERED) return MOE_EINVAL;     // a masked op has nothing to combine
   // after a launch that ran the slot in its paired form, the expert outputs lie in the pair's shared row space
   const int desc = ctx->ran_paired[slot] ? ctx->cfg.max_ops + slot : slot;
   if (launch_combine(ctx->op_dev(desc), ctx->ops[slot].n_tokens, ctx->cfg.top_k, ctx->cfg.hidden,
@@ -427,6 +451,7 @@ int moe_plan_pair(moe_ctx_t* ctx, int slot_prefill, int slot_decode, int carrier
   if (!ctx->planned[sp] || !ctx->planned[sd]) return MOE_ENOTPLANNED;
   const moe_op_t &op = ctx->ops[sp], &od = ctx->ops[sd];
   if (op.cls != MOE_CLASS_PREFILL || od.cls != MOE_CLASS_DECODE) return MOE_EINVAL;
+  if (op.layout != MOE_LAYOUT_GATHERED || od.layout != MOE_LAYOUT_GATHERED) return MOE_EINVAL;
   // one weight tile can only serve rows of both ops if both ops read the same weights
   if (op.w_gate_up != od.w_gate_up || op.w_down != od.w_down || op.s_gate_up != od.s_gate_up || op.s_down != od.s_down)
     return MOE_EINVAL;

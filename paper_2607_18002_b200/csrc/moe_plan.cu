@@ -100,7 +100,7 @@ struct ListScratch {
 // it depends on were claimed long before.
 __device__ __forceinline__ int build_tile_list(int4* tile_list, PlanState* plan, const int* cnt, const int* off, int E,
                                                 int NT1, int NT2, int T, int work_rows, int x_moe, int planned,
-                                                int n_extra_gemm) {
+                                                int n_extra_gemm, int g1_kind = kGateUp) {
   __shared__ ListScratch ls;
   const int e = threadIdx.x;
   const int we = (e < E) ? (cnt[e] + work_rows - 1) / work_rows : 0;
@@ -142,7 +142,7 @@ __device__ __forceinline__ int build_tile_list(int4* tile_list, PlanState* plan,
     const int b1 = ls.g_base1[gi] + ls.moff[x] * NT1, b2 = ls.g_base2[gi] + ls.moff[x] * NT2;
     for (int i = lane; i < wx * NT1; i += 32) {
       const int n = i / wx, j = i - n * wx;
-      tile_list[b1 + i] = make_entry(kGateUp, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
+      tile_list[b1 + i] = make_entry(g1_kind, n, mx + j, ox + j * work_rows, min(work_rows, cx - j * work_rows), x);
     }
     for (int i = lane; i < wx * NT2; i += 32) {
       const int n = i / wx, j = i - n * wx;
@@ -309,6 +309,52 @@ plan_small_kernel(const OpDev* __restrict__ op, Global* g, int slot, int n_chunk
   __threadfence_block();
   __syncthreads();
   if (warp < n_chunks) scatter_chunk(op, R, E, warp, sm + warp * E, lane);
+}
+
+// ---------------------------------------------------------------- masked layout
+// The activations already sit in per-expert slabs of slab_rows rows; counts[e] (an input here) says how many
+// rows of slab e are valid.  Nothing is permuted: the plan is the exclusive prefix sum for `offsets`, the
+// m-tile table (first row of a tile = e * slab_rows + 128 j) and the queue list over the slabs' valid rows.
+__global__ void __launch_bounds__(1024)
+plan_masked_kernel(const OpDev* __restrict__ op, Global* g, int slot, int E, int NT1, int NT2, int slab_rows, int work_rows) {
+  __shared__ int warp_sums[33];
+  __shared__ int s_cnt[kMaxExperts], s_off[kMaxExperts];
+  const int e = threadIdx.x;
+  int cnt = 0;
+  if (e < E) {
+    cnt = op->counts[e];
+    if (cnt < 0 || cnt > slab_rows) {        // a count the slab cannot hold: reported, the slab is left out
+      report(&g->status, MOE_EBOUNDS, slot, e, cnt, 4);
+      cnt = 0;
+    }
+    s_cnt[e] = cnt;
+    s_off[e] = e * slab_rows;
+  }
+  int total;
+  const int off = block_excl_scan(cnt, &total, warp_sums);
+  if (e < E) op->offsets[e] = off;
+  if (e == 0) op->offsets[E] = total;
+  const int me = (e < E) ? (cnt + kTileM - 1) / kTileM : 0;
+  int x_moe;
+  const int m0 = block_excl_scan(me, &x_moe, warp_sums);
+  if (e < E) {
+    for (int j = 0; j < me; ++j) {
+      MTile t;
+      t.expert = e;
+      t.row0 = e * slab_rows + j * kTileM;
+      t.rows = min(kTileM, cnt - j * kTileM);
+      t.pad = 0;
+      op->mtiles[m0 + j] = t;
+    }
+  }
+  __syncthreads();
+  build_tile_list(op->tile_list, op->plan, s_cnt, s_off, E, NT1, NT2, 0, work_rows, x_moe, 1, 0, kGateUpDirect);
+}
+
+cudaError_t launch_plan_masked(const OpDev* d_op, Global* g, int slot, int E, int NT1, int NT2, int slab_rows, int work_rows,
+                               cudaStream_t stream) {
+  plan_masked_kernel<<<1, 1024, 0, stream>>>(d_op, g, slot, E, NT1, NT2, slab_rows, work_rows);
+  return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- the paired form of a decode + prefill op

@@ -78,13 +78,17 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
   const int q = warp & 3, ch = (warp - 8) >> 2;
   const int row = q * 32 + lane;
   const bool valid = row < ti.rows;
-  const bool g1 = ti.kind == kGateUp;
+  const bool g1 = ti.kind != kDown;
   const int HB = a.H / 128, IB = a.I / 128;
   const unsigned lane_addr = tmem + ((unsigned)(q * 32) << 16);
   // scale streams of this row / tile
   const float* sx;
   const float *sw0, *sw1;
-  if (g1) {
+  if (ti.kind == kGateUpDirect) {       // masked layout: the row's scales sit at the row's own index
+    sx = op->x_scale + (size_t)(ti.row0 + (valid ? row : 0)) * HB;
+    sw0 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + ti.n) * HB;
+    sw1 = op->s_gate_up + ((size_t)ti.expert * (2 * IB) + IB + ti.n) * HB;
+  } else if (g1) {
     // the row's activation scales: its own op's, or (paired form) the partner's when the row is tagged so
     int tok = 0;
     const OpDev* src = op;
@@ -317,13 +321,16 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         // Weight tiles by tiled TMA.  The A operand of a down tile is the packed intermediate:
         // consecutive rows, one TMA box (8, 32, 128 or 256 rows high, the smallest that holds
         // the tile's rows); the A operand of a gate/up tile is gathered by the gather warps.
-        const bool g1 = ti.kind == kGateUp;
+        const bool g1 = ti.kind != kDown;                  // gate/up weights
+        const bool gathered = ti.kind == kGateUp;          // activation rows come from the gather warps
+        const bool fromx = ti.kind == kGateUpDirect;       // ... or are consecutive rows of x (masked layout)
         const CUtensorMap* tmw = g1 ? &op->tm_w1 : &op->tm_w2;
         const int wrow0 = g1 ? ti.expert * 2 * args.I + ti.n * kTileN1 : ti.expert * args.H + ti.n * kTileN2;
         const int wrow1 = g1 ? wrow0 + args.I : wrow0 + 128;
         const int box = ti.rows <= 8 ? 8 : (ti.rows <= 32 ? 32 : (ti.rows <= 128 ? 128 : 256));
-        const CUtensorMap* tma = box == 8 ? &op->tm_a8 : (box == 32 ? &op->tm_a32 : (box == 128 ? &op->tm_a128 : &op->tm_a256));
-        const unsigned tx = (unsigned)kBBytes + (g1 ? 0u : (unsigned)(box * kRowBytes));
+        const CUtensorMap* tma = fromx ? (box == 8 ? &op->tm_x8 : (box == 32 ? &op->tm_x32 : (box == 128 ? &op->tm_x128 : &op->tm_x256)))
+                                       : (box == 8 ? &op->tm_a8 : (box == 32 ? &op->tm_a32 : (box == 128 ? &op->tm_a128 : &op->tm_a256)));
+        const unsigned tx = (unsigned)kBBytes + (gathered ? 0u : (unsigned)(box * kRowBytes));
         const int claim_at = min(kClaimAt, ti.kblocks - 1);
         bool fail = false;
         for (int kb = 0; kb < ti.kblocks; ++kb) {
@@ -331,7 +338,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
           {
             const unsigned sA = smem_u32(stages + (size_t)stage * kSB);
             single_issue_kblock(smem_u32(&sc->full[stage]), tx, sA + kBOff, sA + kBOff + kBHalfBytes, tmw, kb * kKb,
-                                wrow0, wrow1, sA, tma, ti.row0, g1 ? 0u : 1u);
+                                wrow0, wrow1, sA, tma, ti.row0, gathered ? 0u : 1u);
           }
           if (++stage == kNS) { stage = 0; ph ^= 1u; }
           if (kb == claim_at)              // claim ahead (never blocks here)
@@ -491,7 +498,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
       if (++islot == kRing) { islot = 0; iph ^= 1u; }
       if (kind == kEnd) break;
       if (kind == kCombine) continue;
-      if (kind == kDown) {             // nothing to gather: hand every stage on empty-handed
+      if (kind != kGateUp) {           // nothing to gather: hand every stage on empty-handed
         bool failed = false;
         for (int kb = 0; kb < kblocks; ++kb, ++kiter) {
           const int stage = (int)(kiter % kNS);
@@ -595,7 +602,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
         bool use[2];
         accs.take(ti.rows, use[0], use[1]);
         const bool pair = use[0] && use[1];
-        const bool g1 = ti.kind == kGateUp;
+        const bool g1 = ti.kind != kDown;
         const int passes = (g1 ? kTileN1 : kTileN2) / 64;      // 32-column passes per warp
         const size_t pitch = (size_t)(g1 ? args.I : args.H) * 2;
 #pragma unroll

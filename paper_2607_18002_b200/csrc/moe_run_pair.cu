@@ -138,14 +138,15 @@ __device__ __forceinline__ LoadPlan make_plan(const RunArgs& a, const OpDev* op,
   LoadPlan p;
   const bool pairT = ti.rows > kTileM;
   const int rpc = pairT ? 128 : 64;
-  p.g1 = ti.kind == kGateUp;
+  p.g1 = ti.kind == kGateUp;                 // activation rows come from the gather warps
+  const bool w1 = ti.kind != kDown;          // gate/up weights
   p.wy1 = -1;
   p.a_boxes = 0;
   p.a_box_rows = 0;
   p.ay = ti.row0 + rank * rpc;
   p.tma = &op->tm_a8;
   unsigned a_bytes = 0;
-  if (p.g1) {
+  if (w1) {
     const int base = ti.expert * 2 * a.I + ti.n * kTileN1;
     if (pairT) {                 // leader: the 128 gate rows, other CTA: the 128 up rows
       p.tmw = &op->tm_w1;
@@ -158,12 +159,16 @@ __device__ __forceinline__ LoadPlan make_plan(const RunArgs& a, const OpDev* op,
   } else {
     p.tmw = &op->tm_w2;
     p.wy0 = ti.expert * a.H + ti.n * kTileN2 + 128 * rank;
+  }
+  if (!p.g1) {
+    // consecutive rows: of the packed intermediate (down tile) or of x itself (masked-layout gate/up tile)
+    const bool fromx = w1;
     const int mine = min(ti.rows - rank * rpc, rpc);
     if (mine > 0) {
-      if (mine <= 8) { p.tma = &op->tm_a8; p.a_boxes = 1; p.a_box_rows = 8; }
-      else if (mine <= 32) { p.tma = &op->tm_a32; p.a_boxes = 1; p.a_box_rows = 32; }
-      else if (pairT) { p.tma = &op->tm_a128; p.a_boxes = 1; p.a_box_rows = 128; }
-      else { p.tma = &op->tm_a32; p.a_boxes = 2; p.a_box_rows = 32; }
+      if (mine <= 8) { p.tma = fromx ? &op->tm_x8 : &op->tm_a8; p.a_boxes = 1; p.a_box_rows = 8; }
+      else if (mine <= 32) { p.tma = fromx ? &op->tm_x32 : &op->tm_a32; p.a_boxes = 1; p.a_box_rows = 32; }
+      else if (pairT) { p.tma = fromx ? &op->tm_x128 : &op->tm_a128; p.a_boxes = 1; p.a_box_rows = 128; }
+      else { p.tma = fromx ? &op->tm_x32 : &op->tm_a32; p.a_boxes = 2; p.a_box_rows = 32; }
       a_bytes = (unsigned)(p.a_boxes * p.a_box_rows * kRowBytes);
     }
   }
@@ -518,7 +523,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
         ++gcount;
         tc_fence_after();
         const bool pairT = ti.rows > kTileM;
-        const bool g1 = ti.kind == kGateUp;
+        const bool g1 = ti.kind != kDown;                     // gate/up tile: SwiGLU, output to A
         const int rpc = pairT ? 128 : 64;
         const int lrow0 = pairT ? q * 32 : (q & 1) * 32;     // first of this warp's rows within the CTA's rows
         const int cg = pairT ? 0 : (q >> 1);                  // which 128 weight rows (M = 128 tiles)

@@ -200,7 +200,7 @@ __device__ inline int try_claim(const RunArgs* a, QueueTables* sc, RunHead* rh, 
   ti.slot = slot;
   ti.tile = (int)local;
   ti.cls = cls;
-  ti.kblocks = ti.kind == kCombine ? 0 : (ti.kind == kGateUp ? a->H : a->I) / a->kb_elems;
+  ti.kblocks = ti.kind == kCombine ? 0 : (ti.kind == kDown ? a->I : a->H) / a->kb_elems;
   return 1;
 }
 
@@ -261,7 +261,7 @@ __device__ inline void claim_static(const RunArgs* a, int unit, TileInfo& ti) {
   ti.slot = slot;
   ti.tile = unit;
   ti.cls = op->cls;
-  ti.kblocks = (ti.kind == kGateUp ? a->H : a->I) / a->kb_elems;
+  ti.kblocks = (ti.kind == kDown ? a->I : a->H) / a->kb_elems;
   ti.t_claim = gtime_ns();
 }
 
@@ -308,7 +308,7 @@ __device__ inline void commit_tile(const Ctx& c, RunHead* rh, const TileInfo& ti
   __threadfence();
   fence_async_proxy();
   const unsigned long long t_commit = a->log_cap > 0 ? gtime_ns() : 0ull;   // before it is published
-  if (ti.kind == kGateUp) atomicAdd(&op->g1_done[ti.m], 1);
+  if (ti.kind == kGateUp || ti.kind == kGateUpDirect) atomicAdd(&op->g1_done[ti.m], 1);
   count_commit(a, op, ti.slot, ti.kind != kCombine);
   // a GEMM entry of a paired decode op carries rows of the prefill op too: it counts for both
   if (op->paired && op->cls == MOE_CLASS_DECODE && ti.kind != kCombine) count_commit(a, &a->ops[op->partner], op->partner, true);

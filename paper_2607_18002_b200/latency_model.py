@@ -7,6 +7,7 @@ on a GPU for a grid of (tokens, active experts) with seeded synthetic routing an
 rows of the paper's "same tokens, different active experts" experiment for this machine.
 
     python -m paper_2607_18002_b200.latency_model          # prints the table and the fit (needs a GPU)
+    python -m paper_2607_18002_b200.latency_model --layouts   # gathered vs masked decode layout (Sections 2.4, 7.4)
 """
 from __future__ import annotations
 
@@ -70,7 +71,69 @@ def sweep(E=256, k=8, H=3072, I=1536, tokens=(32, 128, 512), actives=(8, 16, 32,
     return rows
 
 
+def layout_comparison(E=256, k=8, H=3072, I=1536, tokens=128, actives=(8, 16, 32, 64, 128, 256), reps=12, seed=9,
+                      device="cuda:0"):
+    """The same decode batch through the gathered layout (moe_plan builds the permutation, the kernel gathers token
+    rows, the combine returns token order) and through the masked layout of Section 2.4 (the rows already sit in
+    per-expert slabs, the plan only scans the counts, rows are loaded as boxes, outputs stay in slabs), over a growing
+    number of active experts.  Times are plan + persistent launch in microseconds (CUDA events, median of `reps`, L2
+    flushed in between).  Returns rows of dict(active, x_moe, gathered_us, masked_us, slab_rows)."""
+    import torch
+
+    import paper_2607_18002_b200 as moe
+    from workloads import synth
+
+    spec = synth.Spec("layouts", synth.Shape(E, k, H, I), ((synth.DECODE, tokens),), "uniform", None, 0.02, -1.0, seed)
+    W = synth.make_weights(spec)
+    dev = torch.device(device)
+    w1, w2 = W.w_gate_up.to(dev), W.w_down.to(dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    x, _ = synth.make_x(spec, tokens, 0, 0)
+
+    def timed(ctx, b):
+        ts = []
+        for it in range(reps + 3):
+            flush.fill_(it & 1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            ctx.plan(0, b)
+            ctx.run([0], fuse_combine=True)
+            e1.record()
+            torch.cuda.synchronize()
+            ts.append(1e3 * e0.elapsed_time(e1))
+        ctx.check()
+        return float(np.median(ts[3:]))
+
+    rows = []
+    for A in actives:
+        if A < k or A > E:
+            continue
+        ids, w = synth.route_active_pool(np.random.default_rng([seed, A]), tokens, k, E, A)
+        counts = np.bincount(ids.reshape(-1), minlength=E).astype(np.int32)
+        slab_rows = max(8, -(-int(counts.max()) // 8) * 8)
+        ctx = moe.Context(E, k, H, I, max(tokens, -(-E * slab_rows // k)), 1, device=dev)
+        bg = ctx.bind(synth.DECODE, x.to(dev), torch.from_numpy(ids).to(dev), torch.from_numpy(w).to(dev), w1, w2)
+        t_g = timed(ctx, bg)
+        x_moe = ctx.footprint(0)[0]
+        # the dispatch the masked layout presumes: token rows copied into their experts' slabs, in routing order
+        order = np.argsort(ids.reshape(-1), kind="stable")
+        slab = torch.zeros(E, slab_rows, H, dtype=x.dtype)
+        rank = np.concatenate([np.arange(c) for c in counts])
+        slab[torch.from_numpy(ids.reshape(-1)[order]).long(), torch.from_numpy(rank).long()] = x[torch.from_numpy(order // k).long()]
+        bm = moe.bind_masked_op(synth.DECODE, slab.to(dev), torch.from_numpy(counts).to(dev), w1, w2)
+        t_m = timed(ctx, bm)
+        rows.append(dict(active=int((counts > 0).sum()), x_moe=x_moe, gathered_us=t_g, masked_us=t_m, slab_rows=slab_rows))
+        del ctx
+    return rows
+
+
 def main():
+    import sys
+    if "--layouts" in sys.argv:
+        for r in layout_comparison():
+            print("active experts %3d  x_moe %3d  gathered %8.1f us  masked %8.1f us  (%+.1f us, slabs of %d rows)" %
+                  (r["active"], r["x_moe"], r["gathered_us"], r["masked_us"], r["masked_us"] - r["gathered_us"], r["slab_rows"]))
+        return
     rows = sweep()
     alpha, beta, r2 = fit_affine([r["x_moe"] for r in rows], [r["us"] for r in rows])
     for r in rows:

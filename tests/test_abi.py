@@ -44,7 +44,8 @@ def test_host_side_validation_needs_no_gpu(built):
 
 def test_struct_layouts_match_the_header(built):
     assert ctypes.sizeof(moe.moe_config_t) == 40
-    assert ctypes.sizeof(moe.moe_op_t) == 8 + 15 * 8 + 8 + 8 + 8  # after_op and notify_after share a word; decode_sms + padding
+    # after_op and notify_after share a word; decode_sms + layout, slab_rows + padding
+    assert ctypes.sizeof(moe.moe_op_t) == 8 + 15 * 8 + 8 + 8 + 8 + 8
     assert moe.moe_op_t.notify.offset == 8 + 15 * 8 + 8 and moe.moe_op_t.notify_after.offset == 8 + 15 * 8 + 4
     assert ctypes.sizeof(moe.moe_tile_rec_t) == 32 and moe.TILE_REC_DTYPE.itemsize == 32
 
@@ -61,13 +62,15 @@ def test_binding_structs_match_what_a_c_compiler_makes_of_the_header(tmp_path):
         'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(moe_config_t), sizeof(moe_op_t),\n'
         '  offsetof(moe_op_t, y), offsetof(moe_op_t, ready), offsetof(moe_op_t, after_op),\n'
         '  offsetof(moe_op_t, notify_after), offsetof(moe_op_t, notify), sizeof(moe_tile_rec_t));\n'
-        '  printf("%zu\\n", offsetof(moe_op_t, decode_sms)); return 0; }\n')
+        '  printf("%zu %zu %zu\\n", offsetof(moe_op_t, decode_sms), offsetof(moe_op_t, layout), offsetof(moe_op_t, slab_rows));\n'
+        '  return 0; }\n')
     exe = tmp_path / "layout"
     subprocess.run(["gcc", "-I", inc, "-o", str(exe), str(src)], check=True)
     got = [int(v) for v in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
     o = moe.moe_op_t
     assert got == [ctypes.sizeof(moe.moe_config_t), ctypes.sizeof(o), o.y.offset, o.ready.offset, o.after_op.offset,
-                   o.notify_after.offset, o.notify.offset, ctypes.sizeof(moe.moe_tile_rec_t), o.decode_sms.offset]
+                   o.notify_after.offset, o.notify.offset, ctypes.sizeof(moe.moe_tile_rec_t), o.decode_sms.offset,
+                   o.layout.offset, o.slab_rows.offset]
 
 
 def test_missing_library_fails_loudly(monkeypatch, tmp_path):
