@@ -47,14 +47,14 @@ DEFAULT_STEPS = {"c2": (200, 10), "c3": (30, 5), "c4": (4, 3), "c5": (30, 5), "c
 # save/restore is too large); the full-size figures scale them by the number of active experts, because the
 # traffic is the weights of the active experts, read about once (c3: 256/64, c2: 251/63, c5: 256/32).
 NCU_DRAM_BYTES = {
-    ("c3s", "moe_apk_pair_kernel"): 2.029e9 + 0.160e9,
-    ("c3", "moe_apk_pair_kernel"): (2.029e9 + 0.160e9) * 256 / 64,
-    ("c2s", "moe_apk_pair_kernel"): 1.815e9 + 0.007e9,
-    ("c2", "moe_apk_pair_kernel"): (1.815e9 + 0.007e9) * 251 / 63,
-    ("c4s", "moe_apk_pair_kernel"): 4.036e9 + 0.350e9,
-    ("c4", "moe_apk_pair_kernel"): (4.036e9 + 0.350e9) * 256 / 64,
-    ("c5s", "moe_apk_kernel"): 2.524e9 + 0.087e9,
-    ("c5", "moe_apk_kernel"): (2.524e9 + 0.087e9) * 256 / 32,
+    ("c3s", "moe_apk_pair_kernel"): 2.050e9 + 0.163e9,
+    ("c3", "moe_apk_pair_kernel"): (2.050e9 + 0.163e9) * 256 / 64,
+    ("c2s", "moe_apk_pair_kernel"): 1.816e9 + 0.016e9,
+    ("c2", "moe_apk_pair_kernel"): (1.816e9 + 0.016e9) * 251 / 63,
+    ("c4s", "moe_apk_pair_kernel"): 3.116e9 + 0.337e9,           # decode + prefill op paired (carrier tiles)
+    ("c4", "moe_apk_pair_kernel"): (3.116e9 + 0.337e9) * 256 / 64,
+    ("c5s", "moe_apk_kernel"): 1.743e9 + 0.070e9,                # paired
+    ("c5", "moe_apk_kernel"): (1.743e9 + 0.070e9) * 256 / 32,
 }
 
 def load_peaks():
@@ -682,10 +682,12 @@ def measure(name: str, args, K: int, Wm: int, rank: int, world: int, local: int,
     else:
         roof = {"bound": "tensor", "achieved": flops_launch / t_run / 1e12,
                 "peak": tpeak, "unit": "TFLOP/s", "frac": tensor_frac}
-    roof.update({"traffic": NCU_DRAM_BYTES.get((name, kernel_name)), "kernel": kernel_name,
+    # the captures of the co-scheduled workloads are of the paired form
+    tkey = (name, kernel_name) if (w.pair or len(w.spec.ops) == 1) else None
+    roof.update({"traffic": NCU_DRAM_BYTES.get(tkey), "kernel": kernel_name,
                  "traffic_source": "ncu dram__bytes_read.sum + dram__bytes_write.sum of one launch of the small variant, "
                                    "scaled by active experts (see profiles/)"
-                                   if (name, kernel_name) in NCU_DRAM_BYTES else None,
+                                   if tkey in NCU_DRAM_BYTES else None,
                  "peak_source": peak_src, "peak_kind": "sustained" if long_step else "burst",
                  "launch_ms_mean": 1e3 * t_run, "launch_ms_min": float(np.min(run_ms)),
                  "algorithmic_flops_per_launch": flops_launch,
