@@ -361,9 +361,9 @@ cudaError_t launch_plan_masked(const OpDev* d_op, Global* g, int slot, int E, in
 // Two ops of one launch that share their expert weights can share weight tiles too.  The paired form puts
 // the routed rows of both into ONE packed row space -- per expert the prefill rows (in their plan's order)
 // followed by the decode rows (in theirs) -- and cuts it into two queue lists: per expert, the decode list
-// takes the decode rows plus as many of the prefill rows just before them as fit into the decode rows' last
-// tile of `carrier_rows` rows ("carrier" tiles: claimed with decode priority, they stream a weight tile once
-// for rows of both ops); the prefill list takes the rest.  Nothing about a row's arithmetic depends on the
+// takes the decode rows plus the ragged tail of the prefill rows just before them if it fits into the decode
+// rows' last tile of `carrier_rows` rows ("carrier" tiles: claimed with decode priority, they stream a weight
+// tile once for rows of both ops); the prefill list takes the rest.  Nothing about a row's arithmetic depends on the
 // tile it sits in, so the outputs are those of the unpaired ops, bit for bit.
 //   dp / pp: the paired descriptors (their PlanStates and lists are written here), d / p: the plain ones,
 //   whose counts and offsets the two moe_plan calls have written earlier on the stream.
@@ -375,8 +375,12 @@ plan_pair_kernel(const OpDev* dp, const OpDev* pp, const OpDev* d, const OpDev* 
   if (e < E) {
     const int cd = d->counts[e], cp = p->counts[e];
     const int moff = d->offsets[e] + p->offsets[e];
+    // the carrier takes the ragged tail of the prefill rows (what is left over after the prefill op's full work
+    // tiles) when that tail fits beside the decode rows: a prefill tile less to run.  A tail that does not fit
+    // stays where it is -- moving part of it would make the carrier heavier and save nothing.
     const int room = cd > 0 ? (cd + carrier_rows - 1) / carrier_rows * carrier_rows - cd : 0;
-    const int take = min(cp, room);
+    const int tail = cp % work_rows;
+    const int take = tail <= room ? tail : 0;
     cnt_p[e] = cp - take;
     off_p[e] = moff;
     cnt_d[e] = cd + take;

@@ -7,7 +7,9 @@ sharing it -- the comparison of Section 7.3 of the paper, run on this library's 
   partition   two launches at the same time with disjoint static grids (q CTAs for decode, the
               rest for prefill): what a spatial partition of the SMs gives;
   apk         ONE persistent launch with both operations, tiles claimed from the decode and the
-              prefill queue with a decode budget of q CTAs, work conserving.
+              prefill queue with a decode budget of q CTAs, work conserving;
+  apk_paired  the same launch with the two operations paired (moe_plan_pair): an expert's decode rows
+              travel in carrier tiles of up to 128 / 256 rows together with prefill rows of that expert.
 
 Times are microseconds from the common start: CUDA events for separate launches; for the single
 launch the decode operation's completion comes from the kernel's tile log.
@@ -30,7 +32,7 @@ def _median(v):
     return float(np.median(np.asarray(v, dtype=np.float64)))
 
 
-def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, budgets=(16, 32, 64, 96),
+def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, budgets=(16, 32, 64, 96, 112, 128),
           reps=5, seed=4, device="cuda:0"):
     import torch
 
@@ -94,14 +96,16 @@ def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, b
         c.check()
         return _median(ts[1:])
 
-    def apk(q):
-        c = moe.Context(E, k, H, I, prefill_tokens, 2, tile_log_entries=1 << 16, device=dev)
+    def apk(q, carrier_rows=None):
+        c = moe.Context(E, k, H, I, prefill_tokens + decode_tokens, 2, tile_log_entries=1 << 16, device=dev)
         bp, bd = bind(c, ops[0]), bind(c, ops[1])
         t_all, t_dec = [], []
         for _ in range(reps + 1):
             c.set_budget(q)
             c.plan(0, bp)
             c.plan(1, bd)
+            if carrier_rows:
+                c.plan_pair(0, 1, carrier_rows)
             e0 = torch.cuda.Event(enable_timing=True)
             e1 = torch.cuda.Event(enable_timing=True)
             e0.record()
@@ -126,6 +130,10 @@ def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, b
     for q in budgets:
         ta, td = apk(q)
         rows.append(dict(arm="apk", q=q, prefill_us=ta, decode_us=td))
+    for cr in (128, 256):
+        for q in budgets:
+            ta, td = apk(q, cr)
+            rows.append(dict(arm=f"apk_paired{cr}", q=q, prefill_us=ta, decode_us=td))
     return rows
 
 
@@ -199,7 +207,7 @@ def main():
         return
     rows = study()
     for r in rows:
-        print("%-10s q=%-4s prefill done %9.1f us   decode done %9.1f us" %
+        print("%-13s q=%-4s prefill done %9.1f us   decode done %9.1f us" %
               (r["arm"], "-" if r["q"] is None else r["q"], r["prefill_us"], r["decode_us"]))
     print(json.dumps(rows))
 
