@@ -192,8 +192,16 @@ class Workload:
             if self.fp8:
                 self.bytes_alg += float(active.sum()) * 3 * (sh.H // 128) * (sh.I // 128) * 4
             self.layers.append((ops, bound, host))
-        self.launches_per_step = sum(sum(plan_kernels(o.T, sh.k, sh.E) for o in ops_) + 1 + (1 if self.spec.layers > 1 else 0)
-                                     + (2 if self._pairs(ops_) else 0) for ops_, _, _ in self.layers)
+        self.launches_per_step = sum(sum(plan_kernels(o.T, sh.k, sh.E) for o in ops_) + 1 + (1 if self.budget_for(li_) is not None else 0)
+                                     + (2 if self._pairs(ops_) else 0) for li_, (ops_, _, _) in enumerate(self.layers))
+
+    def budget_for(self, li: int):
+        """Decode SM budget written ahead of layer li's launch (None: the budget word is left alone)."""
+        if self.spec.layers > 1:
+            return synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)]
+        if len(self.spec.ops) > 1:
+            return synth.C5_BUDGET
+        return None
 
     def _pairs(self, ops):
         """(prefill slot, decode slot) of a layer that runs paired, else None."""
@@ -215,8 +223,8 @@ class Workload:
         """Whole hot path for one batch; ev (optional) collects (before_run, after_run) events."""
         ctx = self.ctx
         for li, (ops, bound, _) in enumerate(self.layers):
-            if self.spec.layers > 1:
-                ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
+            if self.budget_for(li) is not None:
+                ctx.set_budget(self.budget_for(li))
             self.plan_layer(ctx, ops, bound)
             if ev is not None:
                 e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -261,8 +269,8 @@ class Workload:
                         b.x_scale.copy_(hs, non_blocking=True)
                     b.topk_ids.copy_(hi, non_blocking=True)
                     b.topk_w.copy_(hw, non_blocking=True)
-                if self.spec.layers > 1:
-                    ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
+                if self.budget_for(li) is not None:
+                    ctx.set_budget(self.budget_for(li))
                 self.plan_layer(ctx, ops, bound)
                 ctx.run(list(range(len(bound))), fuse_combine=True)
                 for b, (_, _, _, hy, _) in zip(bound, host):
@@ -294,8 +302,8 @@ class Workload:
                     e_in.record(self.s_h2d)
                 with torch.cuda.stream(self.s_comp):
                     self.s_comp.wait_event(e_in)
-                    if self.spec.layers > 1:
-                        ctx.set_budget(synth.C4_BUDGETS[li % len(synth.C4_BUDGETS)])
+                    if self.budget_for(li) is not None:
+                        ctx.set_budget(self.budget_for(li))
                     self.plan_layer(ctx, ops_l, bound)
                     ctx.run(list(range(len(bound))), fuse_combine=True)
                     e_run = torch.cuda.Event()
@@ -417,7 +425,7 @@ def tile_stats(w: Workload):
     out = {"per_budget": {}, "paired": bool(w.pair)}
     # the workload's own budgets, then larger ones: the latency of a decode op that streams most experts'
     # weights follows its share of the SMs (and with it of the HBM bandwidth)
-    own = tuple(synth.C4_BUDGETS) if w.spec.layers > 1 else (None,)
+    own = tuple(synth.C4_BUDGETS) if w.spec.layers > 1 else (w.budget_for(0),)
     budgets = own + ((96, 112, 128) if w.spec.layers > 1 else ())
     pooled = {"co": [], "iso": []}
     for bi, q in enumerate(budgets):
@@ -713,7 +721,8 @@ def measure(name: str, args, K: int, Wm: int, rank: int, world: int, local: int,
                       "buffers": "the same X / y buffers every step: the step's 7-10 GB of weights pass through "
                                  "the 126 MB L2 between two uses of a buffer",
                       "replicas": world, "fused_combine": True,
-                      "paired_ops": bool(w.pair and any(w._pairs(o) for o, _, _ in w.layers))},
+                      "paired_ops": bool(w.pair and any(w._pairs(o) for o, _, _ in w.layers)),
+                      "decode_budgets": sorted({w.budget_for(li) for li in range(len(w.layers))} - {None})},
            "clocks": clk.summary(), "gpu_launches": w.launches_per_step * K, "roofline": roof}
     if e2e_out:
         res["e2e"], res["e2e_serial"] = e2e_out, e2e_serial

@@ -24,6 +24,10 @@
  *     kernel that hits one stops claiming tiles and returns -- it never traps or hangs.
  *   - There is no CPU fallback: without a CUDA device every compute entry point fails
  *     with MOE_ECUDA.
+ *   - Debug aid: with MOE_APK_POISON=1 in the environment at moe_create, every moe_run first
+ *     fills the scratch (intermediate and expert-output rows) of its ops with NaN patterns, so
+ *     that a row a launch failed to write shows as NaN in y.  Off by default (it costs two
+ *     large memsets per op and launch).
  */
 #ifndef MOE_APK_H_
 #define MOE_APK_H_

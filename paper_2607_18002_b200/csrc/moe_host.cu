@@ -109,6 +109,7 @@ struct moe_ctx {
   unsigned char* ws;
   int n_ctas, sm_count;
   bool pair_kernel;             // bf16 on an even grid: tiles run on CTA pairs (cta_group::2)
+  bool poison;                  // debug: the scratch of every op of a launch is filled with NaN patterns first
   EncodeTiledFn encode;
   moe_op_t ops[kMaxOps];
   bool planned[kMaxOps];
@@ -215,6 +216,10 @@ int moe_create(const moe_config_t* cfg, void* dev_workspace, size_t bytes, moe_c
   const char* single = getenv("MOE_APK_SINGLE_CTA");
   ctx->pair_kernel = cfg->dtype == MOE_DTYPE_BF16 && ctx->n_ctas >= 2 && ctx->n_ctas % 2 == 0 &&
                      !(single && single[0] == '1');
+  // MOE_APK_POISON=1: a row of the intermediate or of the expert output that a launch fails to write then shows
+  // as NaN in y instead of passing for whatever the previous launch left there
+  const char* poison = getenv("MOE_APK_POISON");
+  ctx->poison = poison && poison[0] == '1';
   ctx->encode = reinterpret_cast<EncodeTiledFn>(fn);
   memset(ctx->planned, 0, sizeof(ctx->planned));
   memset(ctx->uploaded, 0, sizeof(ctx->uploaded));
@@ -387,6 +392,14 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
   a.static_kind = -1;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   if (cudaMemsetAsync(ctx->rh(), 0, ctx->L.runzero_bytes, st) != cudaSuccess) return MOE_ECUDA;
+  if (ctx->poison) {
+    for (int i = 0; i < n_ops; ++i) {
+      unsigned char* sb = ctx->slot_base(slots[i]);
+      const size_t a_bytes = ctx->L.D_off - ctx->L.A_off, d_bytes = ctx->L.mtiles_off - ctx->L.D_off;
+      if (cudaMemsetAsync(sb + ctx->L.A_off, 0xff, a_bytes, st) != cudaSuccess) return MOE_ECUDA;
+      if (cudaMemsetAsync(sb + ctx->L.D_off, 0xff, d_bytes, st) != cudaSuccess) return MOE_ECUDA;
+    }
+  }
   const cudaError_t le = ctx->pair_kernel ? launch_pair(a, ctx->rh(), ctx->n_ctas, st)
                                           : launch_run(a, ctx->rh(), ctx->n_ctas, st);
   if (le != cudaSuccess) return MOE_ECUDA;

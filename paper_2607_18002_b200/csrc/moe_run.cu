@@ -348,7 +348,7 @@ __global__ void __launch_bounds__(kThreads, 1) moe_apk_kernel(const __grid_const
             // takes no waiting: free ring slot, op ready, dependencies already met.
             const OpDev* nop = &args.ops[nx.slot];
             bool can = __all_sync(0xffffffffu, mbar_try(&sc->iempty[islot], iph ^ 1u));
-            if (can && nx_need_ready) can = op_ready(&args, nop);
+            if (can && nx_need_ready) can = __shfl_sync(0xffffffffu, op_ready(&args, nop) ? 1 : 0, 0) != 0;   // lane 0's look
             if (can) {
               int met = 1;
               if (lane == 0) {

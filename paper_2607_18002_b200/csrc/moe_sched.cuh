@@ -157,12 +157,18 @@ __device__ inline int try_claim(const RunArgs* a, QueueTables* sc, RunHead* rh, 
   while (h >= sc->cum[cls][i + 1]) ++i;
   int slot = sc->cls_slot[cls][i];
   const OpDev* op = &a->ops[slot];
-  if (!sc->cls_free[cls][i] && !op_ready(a, op)) return -1;
   const unsigned base = h - sc->cum[cls][i];
-  // The head stands at the op's combine entries while GEMM entries they depend on are still running
-  // (other units hold them; for a paired prefill op, the decode list's carrier tiles): nothing to take here
-  // yet -- the caller turns to the other class instead of holding a combine ticket it cannot run.
-  if (base >= (unsigned)op->plan->n_gemm_tiles && ld_acquire(&op->run->gemm_done) < op_gemm_tiles(op)) return -1;
+  // Everything the warp branches on comes from ONE lane's loads: the lanes of this warp run apart after a
+  // sleep, and words such as an op's done flag or the GEMM counter change between one lane's load and the next's.
+  int takeable = 1;
+  if (lane == 0) {
+    if (!sc->cls_free[cls][i] && !op_ready(a, op)) takeable = 0;
+    // The head stands at the op's combine entries while GEMM entries they depend on are still running
+    // (other units hold them; for a paired prefill op, the decode list's carrier tiles): nothing to take here
+    // yet -- the caller turns to the other class instead of holding a combine ticket it cannot run.
+    else if (base >= (unsigned)op->plan->n_gemm_tiles && ld_acquire(&op->run->gemm_done) < op_gemm_tiles(op)) takeable = 0;
+  }
+  if (__shfl_sync(0xffffffffu, takeable, 0) == 0) return -1;
   // the 32 entries from the head on are fetched while the fetch-add is in flight
   const unsigned n_op = sc->cum[cls][i + 1] - sc->cum[cls][i];
   int4 e = make_int4(0, 0, 0, 0);
@@ -211,10 +217,20 @@ __device__ inline int try_claim(const RunArgs* a, QueueTables* sc, RunHead* rh, 
 __device__ inline int claim_once(const Ctx& c, QueueTables* sc, RunHead* rh, int lane, TileInfo& ti,
                                  bool& need_ready) {
   const RunArgs* a = c.a;
-  const int ab = ld_volatile(&c.st->abort);
-  const int q = ld_volatile(&a->g->budget);
-  const unsigned h0 = *reinterpret_cast<volatile unsigned*>(&rh->heads[0]);
-  const unsigned h1 = *reinterpret_cast<volatile unsigned*>(&rh->heads[1]);
+  // one lane reads the words and the warp takes ITS values: the budget word, the abort word and the heads
+  // change while the kernel runs, and the lanes do not load them at the same instant
+  int ab = 0, q = 0;
+  unsigned h0 = 0, h1 = 0;
+  if (lane == 0) {
+    ab = ld_volatile(&c.st->abort);
+    q = ld_volatile(&a->g->budget);
+    h0 = *reinterpret_cast<volatile unsigned*>(&rh->heads[0]);
+    h1 = *reinterpret_cast<volatile unsigned*>(&rh->heads[1]);
+  }
+  ab = __shfl_sync(0xffffffffu, ab, 0);
+  q = __shfl_sync(0xffffffffu, q, 0);
+  h0 = __shfl_sync(0xffffffffu, h0, 0);
+  h1 = __shfl_sync(0xffffffffu, h1, 0);
   if (ab != 0) return 0;
   const int first = ((int)blockIdx.x < q) ? MOE_CLASS_DECODE : MOE_CLASS_PREFILL;
   need_ready = false;
@@ -228,19 +244,25 @@ __device__ inline int claim_once(const Ctx& c, QueueTables* sc, RunHead* rh, int
   return (r1 == 0 && r2 == 0) ? 0 : -1;
 }
 
-// A ticket that landed in an op that is not ready yet: wait for it (bounded).
+// A ticket that landed in an op that is not ready yet: wait for it (bounded).  Whole warp; lane 0 looks and
+// decides, so that all lanes leave together.
 __device__ inline bool wait_op_ready(const Ctx& c, int lane, const TileInfo& ti) {
   const RunArgs* a = c.a;
   const unsigned long long w0 = gtime_ns();
-  while (!op_ready(a, &a->ops[ti.slot])) {
-    __nanosleep(256);
-    if (aborted(c)) return false;
-    if ((long long)(gtime_ns() - w0) > a->wait_ns) {
-      if (lane == 0) report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, slot_of(a, ti.slot), ti.tile);
-      return false;
+  while (true) {
+    int r = 0;                                   // 1: ready, -1: give up
+    if (lane == 0) {
+      if (op_ready(a, &a->ops[ti.slot])) r = 1;
+      else if (aborted(c)) r = -1;
+      else if ((long long)(gtime_ns() - w0) > a->wait_ns) {
+        report(c.st, MOE_ETIMEOUT, 11, (int)blockIdx.x, slot_of(a, ti.slot), ti.tile);
+        r = -1;
+      }
     }
+    r = __shfl_sync(0xffffffffu, r, 0);
+    if (r != 0) return r > 0;
+    __nanosleep(256);
   }
-  return true;
 }
 
 // The plain (non-persistent) launch: unit `unit` of the grid takes queue entry `unit` of the run's only op
@@ -275,13 +297,17 @@ __device__ inline void claim_next(const Ctx& c, QueueTables* sc, RunHead* rh, in
     if (r == 1) return;
     if (r == 0) break;
     __nanosleep(256);                         // an op exists but is not ready yet
-    if ((it & 15u) == 15u) {
-      const unsigned long long now = gtime_ns();
-      if (t0 == 0) t0 = now;
-      else if ((long long)(now - t0) > c.a->wait_ns) {
-        if (lane == 0) report(c.st, MOE_ETIMEOUT, 1, (int)blockIdx.x, 0, 0);
-        break;
+    if ((it & 15u) == 15u) {                  // lane 0's clock decides for the warp
+      int expired = 0;
+      if (lane == 0) {
+        const unsigned long long now = gtime_ns();
+        if (t0 == 0) t0 = now;
+        else if ((long long)(now - t0) > c.a->wait_ns) {
+          report(c.st, MOE_ETIMEOUT, 1, (int)blockIdx.x, 0, 0);
+          expired = 1;
+        }
       }
+      if (__shfl_sync(0xffffffffu, expired, 0)) break;
     }
   }
   ti.kind = kEnd;

@@ -205,3 +205,18 @@ def test_paired_seeded_random_shapes():
         for b, op in zip(bound, ops):
             check_plan(b, op, E)
             assert_close(b.y.float().cpu().numpy(), oracle.forward(OW, op.x, None, op.ids, op.w)["y"])
+
+
+def test_poisoned_scratch_changes_nothing(monkeypatch):
+    """With MOE_APK_POISON=1 the scratch rows start every launch as NaN patterns: outputs stay bit-identical (every row
+    that is read was written by the same launch), unpaired, paired and in e4m3."""
+    for shape in (SMALL.shape, synth.Shape(8, 2, 512, 256, "fp8")):
+        spec = synth.scaled(SMALL, shape=shape)
+        W = synth.make_weights(spec)
+        ops = synth.make_ops(spec)
+        monkeypatch.delenv("MOE_APK_POISON", raising=False)
+        _, _, y_ref, _ = _both_ways(spec, ops, W, 128, True)
+        monkeypatch.setenv("MOE_APK_POISON", "1")
+        _, bound, y, _ = _both_ways(spec, ops, W, 128, True)
+        for a, b in zip(y_ref, y):
+            assert torch.equal(a, b) and torch.isfinite(b.float()).all()

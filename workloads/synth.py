@@ -102,6 +102,7 @@ SPECS["c5s"] = dataclasses.replace(SPECS["c5"], name="c5s", shape=Shape(32, 8, 6
                                    ops=((PREFILL, 512), (DECODE, 64)))
 del scaled_
 C4_BUDGETS = (16, 32, 64)     # decode SM budget cycled between layers
+C5_BUDGET = 96                # decode SM budget of the single co-scheduled FP8 launch (the config names none)
 
 
 def scaled(spec: Spec, **kw) -> Spec:
