@@ -53,8 +53,8 @@ NCU_DRAM_BYTES = {
     ("c2", "moe_apk_pair_kernel"): (1.816e9 + 0.016e9) * 251 / 63,
     ("c4s", "moe_apk_pair_kernel"): 3.116e9 + 0.337e9,           # decode + prefill op paired (carrier tiles)
     ("c4", "moe_apk_pair_kernel"): (3.116e9 + 0.337e9) * 256 / 64,
-    ("c5s", "moe_apk_kernel"): 1.743e9 + 0.070e9,                # paired
-    ("c5", "moe_apk_kernel"): (1.743e9 + 0.070e9) * 256 / 32,
+    ("c5s", "moe_apk_kernel"): 1.570e9 + 0.062e9,                # paired, decode budget 96
+    ("c5", "moe_apk_kernel"): (1.570e9 + 0.062e9) * 256 / 32,
 }
 
 def load_peaks():

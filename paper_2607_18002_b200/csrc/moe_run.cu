@@ -133,19 +133,19 @@ __device__ __forceinline__ bool epilogue_fp8(const Ctx& c, SharedCtl* sc, OpDev*
     if (!__all_sync(0xffffffffu, mbar_wait_inline(c, &sc->pfull[pb], (eph >> pb) & 1u, 19))) return false;
     eph ^= 1u << pb;
     tc_fence_after();
-    // eight 16-column chunks (four per half); the load of chunk c+1 is in flight while chunk c
-    // is multiplied in
+    // four 32-column chunks (two per half), one TMEM load each: tcgen05.wait::ld waits for every load of the
+    // thread, so a second load in flight only ever overlapped one chunk's FMAs; fewer, wider loads are faster
+    // (the other warp of the scheduler partition fills the wait)
     const unsigned pbase = lane_addr + (unsigned)(pb * 256 + ch * 64);
-    unsigned p[2][16];
-    tc_ld16(pbase, p[0]);
+    unsigned p[32];
 #pragma unroll
-    for (int cc = 0; cc < 8; ++cc) {
+    for (int cc = 0; cc < 4; ++cc) {
+      tc_ld32(pbase + (unsigned)((cc >> 1) * 128 + (cc & 1) * 32), p);
       tc_wait_ld();
-      if (cc + 1 < 8) tc_ld16(pbase + (unsigned)(((cc + 1) >> 2) * 128 + ((cc + 1) & 3) * 16), p[(cc + 1) & 1]);
-      const float s = (cc >> 2) ? s1 : s0;
+      const float s = (cc >> 1) ? s1 : s0;
 #pragma unroll
-      for (int i = 0; i < 16; ++i)
-        acc[cc * 16 + i] = fmaf(__uint_as_float(p[cc & 1][i]), s, acc[cc * 16 + i]);
+      for (int i = 0; i < 32; ++i)
+        acc[cc * 32 + i] = fmaf(__uint_as_float(p[i]), s, acc[cc * 32 + i]);
     }
     tc_fence_before();
     __syncwarp();                                 // every lane's TMEM loads have completed
