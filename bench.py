@@ -527,7 +527,7 @@ def persistent_layers(w: Workload, steps: int, warmup: int):
     separate budget write between layers.  Same inputs, same plan calls as the per-layer step."""
     moe, sh = w.moe, w.sh
     n_layers = len(w.layers)
-    ctx = moe.Context(sh.E, sh.k, sh.H, sh.I, max(T for _, T in w.spec.ops), max_ops=2 * n_layers,
+    ctx = moe.Context(sh.E, sh.k, sh.H, sh.I, w.max_tokens, max_ops=2 * n_layers,
                       dtype=moe.MOE_DTYPE_FP8_E4M3 if w.fp8 else moe.MOE_DTYPE_BF16, device=w.device)
     bound = []
     for l, (ops, b_old, _) in enumerate(w.layers):
@@ -542,6 +542,10 @@ def persistent_layers(w: Workload, steps: int, warmup: int):
     def step():
         for s_, b in enumerate(bound):
             ctx.plan(s_, b)
+        for l, (ops, _, _) in enumerate(w.layers):         # the two ops of a layer paired, as in the per-layer step
+            pr = w._pairs(ops)
+            if pr:
+                ctx.plan_pair(2 * l + pr[0], 2 * l + pr[1], 0)
         ctx.run(slots, fuse_combine=True)
 
     for _ in range(warmup):
@@ -567,7 +571,8 @@ def persistent_layers(w: Workload, steps: int, warmup: int):
     same = all(torch.equal(b.y, bo.y) for b, (_, b_old, _) in zip([bound[i:i + 2] for i in range(0, len(bound), 2)], w.layers)
                for b, bo in zip(b, b_old)) if all(len(x[1]) == 2 for x in w.layers) else None
     return {"ms_per_step": ms, "value": w.flops / (ms / 1e3) / 1e12, "unit": UNIT, "ops_in_launch": len(bound),
-            "launches_per_step": sum(plan_kernels(o.T, sh.k, sh.E) for ops_, _, _ in w.layers for o in ops_) + 1,
+            "launches_per_step": sum(plan_kernels(o.T, sh.k, sh.E) for ops_, _, _ in w.layers for o in ops_) + 1
+                                 + sum(2 for ops_, _, _ in w.layers if w._pairs(ops_)),
             "outputs_equal_per_layer_launches": same,
             "per_layer_launches_ms_per_step_alternating": float(np.mean(t_per))}
 

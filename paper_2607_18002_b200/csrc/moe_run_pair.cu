@@ -450,7 +450,7 @@ moe_apk_pair_kernel(const __grid_constant__ RunArgs args, RunHead* rh) {
         const bool theirs = tag != own_tag;
         // an index the plan never wrote is reported below and its row is skipped
         const bool in_range = v >= 0 && (tag == own_tag || tag == partner_tag) && flat < (theirs ? n_rows_p : n_rows);
-        bad |= !in_range;
+        bad |= mine && !in_range;
         tok[j] = (mine && in_range) ? (theirs ? ~(flat / args.k) : flat / args.k) : INT_MIN;
       }
       if (bad) report(c.st, MOE_EBOUNDS, slot_of(&args, slot), row0, rows, 0);

@@ -220,3 +220,42 @@ def test_poisoned_scratch_changes_nothing(monkeypatch):
         _, bound, y, _ = _both_ways(spec, ops, W, 128, True)
         for a, b in zip(y_ref, y):
             assert torch.equal(a, b) and torch.isfinite(b.float()).all()
+
+
+def test_three_paired_layers_in_one_launch():
+    """Six operations in one launch, chained by after_op (prefill l and decode l after prefill l-1), the two ops of
+    every layer paired: results equal the per-layer unpaired launches bit for bit."""
+    shape = synth.Shape(32, 4, 1024, 512)
+    spec = synth.Spec("layersp", shape, ((synth.PREFILL, 1024), (synth.DECODE, 64)), "zipf", 1.0, 1.0, -1.0, 43, layers=3)
+    W = weights_to(synth.make_weights(spec))
+    small = make_ctx(spec, max_tokens=1024, max_ops=2)
+    y_ref = []
+    for l in range(3):
+        b = bind_ops(small, synth.make_ops(spec, l), W)
+        for s_, x in enumerate(b):
+            small.plan(s_, x)
+        small.run([0, 1], fuse_combine=True)
+        small.check()
+        y_ref.append([x.y.clone() for x in b])
+    ctx = make_ctx(spec, max_tokens=1024 + 64, max_ops=6, tile_log_entries=1 << 15)
+    from gpu_util import upload
+    bound = []
+    for l in range(3):
+        for op in synth.make_ops(spec, l):
+            d = upload(op, None, "cuda:0")
+            bound.append(ctx.bind(op.cls, d["x"], d["ids"], d["w"], W.w_gate_up, W.w_down,
+                                  after_op=(2 * (l - 1) if l > 0 else -1),
+                                  decode_sms=((16, 32, 64)[l] if op.cls == synth.DECODE else 0)))
+    for s_, b in enumerate(bound):
+        ctx.plan(s_, b)
+    for l in range(3):
+        ctx.plan_pair(2 * l, 2 * l + 1, (128, 256, 0)[l])
+    ctx.run(list(range(6)), fuse_combine=True)
+    ctx.check()
+    for l in range(3):
+        assert torch.equal(bound[2 * l].y, y_ref[l][0]) and torch.equal(bound[2 * l + 1].y, y_ref[l][1])
+    log = ctx.tile_log()
+    for l in (1, 2):
+        done_prev = log["t_commit"][log["slot"] == 2 * (l - 1)].max()
+        assert log["t_commit"][log["slot"] == 2 * l].min() >= done_prev
+        assert log["t_commit"][log["slot"] == 2 * l + 1].min() >= done_prev
