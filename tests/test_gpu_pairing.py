@@ -222,10 +222,11 @@ def test_poisoned_scratch_changes_nothing(monkeypatch):
             assert torch.equal(a, b) and torch.isfinite(b.float()).all()
 
 
-def test_three_paired_layers_in_one_launch():
+@pytest.mark.parametrize("dtype", ["bf16", "fp8"])
+def test_three_paired_layers_in_one_launch(dtype):
     """Six operations in one launch, chained by after_op (prefill l and decode l after prefill l-1), the two ops of
     every layer paired: results equal the per-layer unpaired launches bit for bit."""
-    shape = synth.Shape(32, 4, 1024, 512)
+    shape = synth.Shape(32, 4, 1024, 512, dtype)
     spec = synth.Spec("layersp", shape, ((synth.PREFILL, 1024), (synth.DECODE, 64)), "zipf", 1.0, 1.0, -1.0, 43, layers=3)
     W = weights_to(synth.make_weights(spec))
     small = make_ctx(spec, max_tokens=1024, max_ops=2)
@@ -243,13 +244,14 @@ def test_three_paired_layers_in_one_launch():
     for l in range(3):
         for op in synth.make_ops(spec, l):
             d = upload(op, None, "cuda:0")
-            bound.append(ctx.bind(op.cls, d["x"], d["ids"], d["w"], W.w_gate_up, W.w_down,
+            bound.append(ctx.bind(op.cls, d["x"], d["ids"], d["w"], W.w_gate_up, W.w_down, x_scale=d["x_scale"],
+                                  s_gate_up=W.s_gate_up, s_down=W.s_down,
                                   after_op=(2 * (l - 1) if l > 0 else -1),
                                   decode_sms=((16, 32, 64)[l] if op.cls == synth.DECODE else 0)))
     for s_, b in enumerate(bound):
         ctx.plan(s_, b)
     for l in range(3):
-        ctx.plan_pair(2 * l, 2 * l + 1, (128, 256, 0)[l])
+        ctx.plan_pair(2 * l, 2 * l + 1, 128 if dtype == "fp8" else (128, 256, 0)[l])
     ctx.run(list(range(6)), fuse_combine=True)
     ctx.check()
     for l in range(3):
