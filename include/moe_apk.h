@@ -170,7 +170,8 @@ int moe_run(moe_ctx_t* ctx, const int32_t* slots, int n_ops, int fuse_combine, v
  * w_down / scale pointers) so that a launch running both streams an expert's weight tile ONCE for rows of
  * both: the decode op's rows of an expert travel in "carrier" tiles together with the ragged tail of that
  * expert's prefill rows (what its full prefill tiles leave over) when the tail fits into the decode rows'
- * last tile of `carrier_rows` rows (128, or 256 for bf16; 0 = the largest).  Carrier tiles belong to the decode class -- decode priority and the budget work as before
+ * last tile of `carrier_rows` rows (128 or 256; 0 = the kernel's work-tile height: 256 for bf16, 128 for e4m3,
+ * where a 256-row carrier runs as two 128-row tiles that follow one another).  Carrier tiles belong to the decode class -- decode priority and the budget work as before
  * (Sections 4.2, 6.4) -- and the prefill op keeps the remaining rows.  A row's arithmetic does not depend
  * on the tile it sits in, so y of both ops is bit-identical to the unpaired launch; counts, offsets and the
  * permutations of moe_plan are untouched (the shared row space is private workspace).

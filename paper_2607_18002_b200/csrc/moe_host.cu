@@ -470,7 +470,7 @@ int moe_plan_pair(moe_ctx_t* ctx, int slot_prefill, int slot_decode, int carrier
     return MOE_EINVAL;
   const bool fp8 = c.dtype == MOE_DTYPE_FP8_E4M3;
   if (carrier_rows == 0) carrier_rows = fp8 ? kWorkRowsFp8 : kWorkRowsBf16;
-  if (carrier_rows != 128 && !(carrier_rows == 256 && !fp8)) return MOE_EINVAL;
+  if (carrier_rows != 128 && carrier_rows != 256) return MOE_EINVAL;
   const Layout& L = ctx->L;
   const long long Rp = (long long)op.n_tokens * c.top_k, Rd = (long long)od.n_tokens * c.top_k;
   if (Rp + Rd > L.max_rows) return MOE_ENOSPC;      // the shared row space lives in one slot's scratch

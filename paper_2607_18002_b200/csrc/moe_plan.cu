@@ -379,7 +379,7 @@ plan_pair_kernel(const OpDev* dp, const OpDev* pp, const OpDev* d, const OpDev* 
     // tiles) when that tail fits beside the decode rows: a prefill tile less to run.  A tail that does not fit
     // stays where it is -- moving part of it would make the carrier heavier and save nothing.
     const int room = cd > 0 ? (cd + carrier_rows - 1) / carrier_rows * carrier_rows - cd : 0;
-    const int tail = cp % work_rows;
+    const int tail = cp % max(work_rows, carrier_rows);
     const int take = tail <= room ? tail : 0;
     cnt_p[e] = cp - take;
     off_p[e] = moff;
@@ -388,8 +388,9 @@ plan_pair_kernel(const OpDev* dp, const OpDev* pp, const OpDev* d, const OpDev* 
   }
   __syncthreads();
   const int ok = (d->plan->planned && p->plan->planned) ? 1 : 0;
-  const int n_dec = build_tile_list(dp->tile_list, dp->plan, cnt_d, off_d, E, NT1, NT2, d->n_tokens, carrier_rows,
-                                    d->plan->n_mtiles, ok, 0);
+  // a carrier taller than the kernel's work tile (e4m3: 128 rows) is cut into work tiles that follow one another
+  const int n_dec = build_tile_list(dp->tile_list, dp->plan, cnt_d, off_d, E, NT1, NT2, d->n_tokens,
+                                    min(carrier_rows, work_rows), d->plan->n_mtiles, ok, 0);
   // every GEMM entry of the decode list may carry prefill rows: the prefill op is complete when they are too
   build_tile_list(pp->tile_list, pp->plan, cnt_p, off_p, E, NT1, NT2, p->n_tokens, work_rows, p->plan->n_mtiles, ok,
                   n_dec);

@@ -180,12 +180,13 @@ def test_paired_fp8_equals_unpaired_and_mirrored_oracle(shape):
     spec = synth.Spec("fp8p", shape, ((synth.PREFILL, 300), (synth.DECODE, 37)), "softmax_topk", None, 1.0, -1.0, 35)
     W = synth.make_weights(spec)
     ops = synth.make_ops(spec)
-    ctx, bound, _, _ = _both_ways(spec, ops, W, 128, True)
     OW = oracle_weights(spec, W)
-    for b, op in zip(bound, ops):
-        check_plan(b, op, shape.E)
-        ref = oracle.forward(OW, op.x, op.x_scale, op.ids, op.w, round_A=oracle.ROUND_E4M3_1X128)
-        assert_close(b.y.float().cpu().numpy(), ref["y"], atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
+    for carrier_rows in (128, 256):                   # 256: the carrier runs as two 128-row tiles
+        ctx, bound, _, _ = _both_ways(spec, ops, W, carrier_rows, True)
+        for b, op in zip(bound, ops):
+            check_plan(b, op, shape.E)
+            ref = oracle.forward(OW, op.x, op.x_scale, op.ids, op.w, round_A=oracle.ROUND_E4M3_1X128)
+            assert_close(b.y.float().cpu().numpy(), ref["y"], atol=ATOL8, rtol=RTOL8, rel_l2=REL_L2_8)
 
 
 def test_paired_seeded_random_shapes():
