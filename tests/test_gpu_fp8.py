@@ -18,10 +18,10 @@ from gpu_util import (ATOL8, REL_L2_8, RTOL8, assert_close, bind_ops, check_plan
 pytestmark = pytest.mark.gpu
 
 
-def _run(spec, ops=None, W=None, budget=None):
+def _run(spec, ops=None, W=None, budget=None, pair=False):
     W = W or synth.make_weights(spec)
     ops = ops or synth.make_ops(spec)
-    ctx = make_ctx(spec, max_tokens=max(o.T for o in ops), max_ops=len(ops))
+    ctx = make_ctx(spec, max_tokens=sum(o.T for o in ops) if pair else max(o.T for o in ops), max_ops=len(ops))
     bound = bind_ops(ctx, ops, weights_to(W))
     if budget is not None:
         ctx.set_budget(budget)
@@ -29,6 +29,15 @@ def _run(spec, ops=None, W=None, budget=None):
         ctx.plan(s, b)
     ctx.run(list(range(len(bound))), fuse_combine=True)
     ctx.check()
+    if pair:            # the same launch with the prefill op (slot 0) and the decode op (slot 1) paired: same bits
+        y = [b.y.clone() for b in bound]
+        for s, b in enumerate(bound):
+            b.y.zero_()
+            ctx.plan(s, b)
+        ctx.plan_pair(0, 1, 0)
+        ctx.run(list(range(len(bound))), fuse_combine=True)
+        ctx.check()
+        assert all(torch.equal(a, b.y) for a, b in zip(y, bound))
     return ctx, bound, ops, W
 
 
@@ -168,7 +177,7 @@ def test_c5_full_size_sampled():
     below a recorded ceiling, so that it cannot grow unnoticed."""
     spec = synth.SPECS["c5"]
     W = synth.make_weights(spec, threads=16)
-    ctx, bound, ops, _ = _run(spec, W=W, budget=32)
+    ctx, bound, ops, _ = _run(spec, W=W, budget=synth.C5_BUDGET, pair=True)    # unpaired, then paired as the bench runs it
     OW = oracle_weights(spec, W)
     for b, op in zip(bound, ops):
         check_plan(b, op, spec.shape.E)

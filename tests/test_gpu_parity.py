@@ -564,11 +564,11 @@ def test_c3_full_size_sampled(big_weights, fuse):
 
 
 def test_c4_full_size_layers_budgets_and_both_weight_sets():
-    """C4 as the bench runs it: layer 0 at decode budgets 16 and 64 (bit-identical outputs), layer 1 at
-    budget 32 on the second weight set; on each the oracle evaluates every decode token, the rows at every
-    expert-segment edge of the prefill op and a seeded token sample."""
+    """C4 as the bench runs it: layer 0 at decode budgets 16 and 64, layer 1 at budget 32 on the second weight
+    set, each also with the two ops paired (all outputs of a layer bit-identical); on each layer the oracle
+    evaluates every decode token, the rows at every expert-segment edge of the prefill op and a seeded sample."""
     spec = synth.SPECS["c4"]
-    ctx = make_ctx(spec)
+    ctx = make_ctx(spec, max_tokens=sum(T for _, T in spec.ops))      # room for the paired form's shared row space
     for layer, budgets in ((0, (16, 64)), (1, (32,))):
         W = synth.make_weights(spec, layer=layer, threads=16)
         Wd = weights_to(W)
@@ -585,6 +585,15 @@ def test_c4_full_size_layers_budgets_and_both_weight_sets():
             ctx.run([0, 1], fuse_combine=True)
             ctx.check()
             ys.append([b.y.clone() for b in bound])
+        # the launch as the bench times it: the two ops paired (carrier tiles), same budget
+        for b in bound:
+            b.y.zero_()
+        for s, b in enumerate(bound):
+            ctx.plan(s, b)
+        ctx.plan_pair(0, 1, 0)
+        ctx.run([0, 1], fuse_combine=True)
+        ctx.check()
+        ys.append([b.y.clone() for b in bound])
         for other in ys[1:]:
             assert all(torch.equal(a, b) for a, b in zip(ys[0], other))
         _check_sampled(ctx, spec, bound, ops, OW, n_extra=96, cap=640)
