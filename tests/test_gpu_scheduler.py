@@ -233,3 +233,54 @@ def test_plain_launches_give_the_same_bits_as_the_persistent_kernel():
     rows = scheduler_overhead(E=32, k=4, H=1024, I=512, prefill_tokens=2048, zipf_s=1.0, decode_tokens=32,
                               actives=(8, 32), reps=3)
     assert len(rows) == 3 and all(r["same_bits"] and r["persistent_us"] > 0 and r["plain_us"] > 0 for r in rows)
+
+
+def test_a_whole_layer_step_replays_from_a_cuda_graph():
+    """Every call of a layer step only enqueues work (a 4-byte budget write, the plan kernels, the pairing, the
+    persistent launch), so the step can be captured once and replayed without the host touching it again -- the
+    property the paper's kernel is built around (Section 4.2: no CPU reconfiguration between layers).  New routing
+    written into the same buffers is picked up by the replay."""
+    spec = synth.Spec("graph", SPEC.shape, ((synth.PREFILL, 1500), (synth.DECODE, 48)), "zipf", 1.0, 1.0, -1.0, 45, layers=2)
+    W = weights_to(synth.make_weights(spec))
+    ctx = make_ctx(spec, max_tokens=1548, max_ops=2)
+    ops0, ops1 = synth.make_ops(spec, 0), synth.make_ops(spec, 1)
+    bound = bind_ops(ctx, ops0, W)
+
+    def step():
+        ctx.set_budget(32)
+        ctx.plan(0, bound[0])
+        ctx.plan(1, bound[1])
+        ctx.plan_pair(0, 1, 0)
+        ctx.run([0, 1], fuse_combine=True)
+
+    step()                                     # first calls upload the descriptors: keep them out of the capture
+    ctx.check()
+    y0 = [b.y.clone() for b in bound]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(g, stream=side):
+            step()
+    torch.cuda.current_stream().wait_stream(side)
+    for b in bound:
+        b.y.zero_()
+    g.replay()
+    ctx.check()
+    assert all(torch.equal(a, b.y) for a, b in zip(y0, bound))
+    # other inputs in the same buffers: the replay plans and runs them
+    from gpu_util import upload
+    for b, op in zip(bound, ops1):
+        d = upload(op, None, "cuda:0")
+        b.x.copy_(d["x"]); b.topk_ids.copy_(d["ids"]); b.topk_w.copy_(d["w"])
+    g.replay()
+    ctx.check()
+    y_graph = [b.y.clone() for b in bound]
+    step()
+    ctx.check()
+    assert all(torch.equal(a, b.y) for a, b in zip(y_graph, bound))
+    import oracle
+    from gpu_util import assert_close, oracle_weights
+    OW = oracle_weights(spec, synth.make_weights(spec))
+    for b, op in zip(bound, ops1):
+        assert_close(b.y.float().cpu().numpy(), oracle.forward(OW, op.x, None, op.ids, op.w)["y"])
