@@ -18,7 +18,9 @@
  * Parity pins (see tests/test_oracle_pins.py): the plan equals a stable argsort
  * and a brute-force rescan; the FFN equals a float64 library MLP for E=1,k=1;
  * the whole equals dense every-expert evaluation in float64; e4m3 decode equals
- * the library's table for all 256 codes.  The paper prints no worked numeric
+ * the library's table for all 256 codes; the rounding switches of the FFN (e4m3 per
+ * row and 128 columns, bf16 of the intermediate, bf16 of the output) equal the
+ * library casts applied to the un-rounded values.  The paper prints no worked numeric
  * example of this path, so numeric parity against the paper itself is unpinned.
  */
 #include <math.h>
