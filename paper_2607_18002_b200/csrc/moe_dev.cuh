@@ -17,7 +17,9 @@ constexpr int kTileN2 = 256;         // output columns per down-GEMM tile
 constexpr int kBlockK = 64;          // K elements per pipeline stage (one 128-byte swizzle row of bf16)
 constexpr int kRowBytes = kBlockK * 2;
 constexpr int kStages = 3;           // shared-memory pipeline depth (64 KB per stage)
-constexpr int kCombineTokens = 16;   // tokens per combine tile
+constexpr int kCombineTokens = 16;   // tokens per combine tile ...
+constexpr int kCombineTokensSmall = 4;     // ... of an op with at most kCombineSmallBatch tokens (a decode batch): its
+constexpr int kCombineSmallBatch = 1024;   // combine is a latency chain per token, so it is spread over more units
 constexpr int kPlanChunk = 256;      // routed rows ranked by one warp in the plan kernels
 constexpr int kGroupWork = 16;       // work tiles per dependency group of the tile list
 constexpr int kWorkRowsBf16 = 256;   // rows of a work tile: two m-tiles share each weight tile
@@ -27,6 +29,8 @@ constexpr int kMaxExperts = 1024;
 
 // kGateUpDirect: a gate/up tile whose activation rows are consecutive rows of x (masked layout): they are
 // loaded by TMA like the rows of a down tile instead of being gathered through a permutation
+__host__ __device__ inline int combine_tile_tokens(int T) { return T <= kCombineSmallBatch ? kCombineTokensSmall : kCombineTokens; }
+
 enum TileKind : int { kGateUp = 0, kDown = 1, kCombine = 2, kGateUpDirect = 3 };
 
 // Queue entry (16 bytes, one load per claim): x = kind | n-tile << 4 | m-tile << 12,

@@ -66,7 +66,11 @@ Layout make_layout(const moe_config_t* c) {
   L.max_mtiles = (L.max_rows + kTileM - 1) / kTileM + c->n_experts;
   L.NT1 = (int)(I / kTileN1);
   L.NT2 = (int)(H / kTileN2);
-  const int max_comb = (c->max_tokens_per_op + kCombineTokens - 1) / kCombineTokens;
+  // combine entries of the largest op: small batches use smaller combine tiles
+  const int small_t = c->max_tokens_per_op < kCombineSmallBatch ? c->max_tokens_per_op : kCombineSmallBatch;
+  const int comb_small = (small_t + kCombineTokensSmall - 1) / kCombineTokensSmall;
+  const int comb_large = (c->max_tokens_per_op + kCombineTokens - 1) / kCombineTokens;
+  const int max_comb = comb_small > comb_large ? comb_small : comb_large;
   L.max_tiles = L.max_mtiles * (L.NT1 + L.NT2) + max_comb;
   const size_t n_chunks = ((size_t)L.max_rows + kPlanChunk - 1) / kPlanChunk;
 

@@ -150,9 +150,10 @@ __device__ __forceinline__ int build_tile_list(int4* tile_list, PlanState* plan,
     }
   }
   const int n_gemm = ls.ntiles;
-  const int n_comb = (T + kCombineTokens - 1) / kCombineTokens;
+  const int ct = combine_tile_tokens(T);
+  const int n_comb = (T + ct - 1) / ct;
   for (int c = threadIdx.x; c < n_comb; c += blockDim.x)
-    tile_list[n_gemm + c] = make_entry(kCombine, 0, c, c * kCombineTokens, min(kCombineTokens, T - c * kCombineTokens), 0);
+    tile_list[n_gemm + c] = make_entry(kCombine, 0, c, c * ct, min(ct, T - c * ct), 0);
   if (threadIdx.x == 0) {
     PlanState ps;
     ps.n_mtiles = x_moe;

@@ -13,6 +13,12 @@ ATOL, RTOL, REL_L2 = 1e-2, 1e-2, 5e-3
 ATOL8, RTOL8, REL_L2_8 = 4e-2, 4e-2, 3e-2
 
 
+def n_combine_tiles(T: int) -> int:
+    """Combine entries of an op's queue list: 16 tokens per tile, 4 for a batch of at most 1024 tokens."""
+    ct = 4 if T <= 1024 else 16
+    return -(-T // ct)
+
+
 def upload(op: synth.Op, W: synth.Weights, dev="cuda:0"):
     t = lambda a: None if a is None else (a if isinstance(a, torch.Tensor) else torch.from_numpy(a)).to(dev)
     return dict(x=t(op.x), x_scale=t(op.x_scale), ids=t(op.ids), w=t(op.w))

@@ -9,7 +9,7 @@ import oracle
 import paper_2607_18002_b200 as moe
 from workloads import synth
 
-from gpu_util import (assert_close, bind_ops, check_plan, check_tiles, make_ctx, oracle_weights,
+from gpu_util import (assert_close, bind_ops, check_plan, check_tiles, make_ctx, n_combine_tiles, oracle_weights,
                       weights_to)
 
 pytestmark = pytest.mark.gpu
@@ -409,7 +409,7 @@ def test_several_free_ops_of_each_class_in_one_run(fuse, n_ctas):
     log = ctx.tile_log()
     OW = oracle_weights(spec, W)
     for s, (b, op) in enumerate(zip(bound, ops)):
-        n = ctx.footprint(s)[1] - (0 if fuse else -(-op.T // 16))     # unfused: no combine tiles in the launch
+        n = ctx.footprint(s)[1] - (0 if fuse else n_combine_tiles(op.T))     # unfused: no combine tiles in the launch
         assert sorted(log["tile"][log["slot"] == s].tolist()) == list(range(n))      # every entry exactly once
         assert_close(b.y.float().cpu().numpy(), oracle.forward(OW, op.x, None, op.ids, op.w)["y"])
 

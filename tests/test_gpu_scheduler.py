@@ -8,7 +8,7 @@ import torch
 import paper_2607_18002_b200 as moe
 from workloads import synth
 
-from gpu_util import bind_ops, make_ctx, weights_to
+from gpu_util import bind_ops, make_ctx, n_combine_tiles, weights_to
 
 pytestmark = pytest.mark.gpu
 
@@ -41,7 +41,7 @@ def test_every_entry_once_and_dependencies_hold():
         # a combine tile is published only after the op's last GEMM tile committed; with
         # claim-ahead it may have been *claimed* earlier, so compare commits
         assert g["t_commit"][g["kind"] == 2].min() >= last_gemm
-        assert len(first_combine) == -(-SPEC.ops[slot][1] // 16)
+        assert len(first_combine) == n_combine_tiles(SPEC.ops[slot][1])
     assert np.all(log["t_commit"] >= log["t_claim"])
 
 
@@ -221,7 +221,7 @@ def test_plain_launches_give_the_same_bits_as_the_persistent_kernel():
         ctx.check()
         assert torch.equal(y, b.y)
         log = ctx.tile_log()                   # every GEMM entry exactly once, by the unit with its index
-        n_gemm = ctx.footprint(s_)[1] - -(-op.T // 16)
+        n_gemm = ctx.footprint(s_)[1] - n_combine_tiles(op.T)
         assert sorted(log["tile"].tolist()) == list(range(n_gemm))
         assert np.array_equal(log["cta"] // 2, log["tile"])
     single = make_ctx(SPEC, max_tokens=4096, max_ops=1, n_ctas=3)          # single-CTA kernel: no plain form
