@@ -6,6 +6,9 @@ sharing it -- the comparison of Section 7.3 of the paper, run on this library's 
               right after the prefill one: launch-granularity sharing, no preemption;
   partition   two launches at the same time with disjoint static grids (q CTAs for decode, the
               rest for prefill): what a spatial partition of the SMs gives;
+  green       the same two launches, each on a stream of its own CUDA green context whose SM set the
+              driver enforces (q SMs for decode, the remaining SMs for prefill); left out with the
+              driver's answer if green contexts cannot be made here;
   apk         ONE persistent launch with both operations, tiles claimed from the decode and the
               prefill queue with a decode budget of q CTAs, work conserving;
   apk_paired  the same launch with the two operations paired (moe_plan_pair): an expert's decode rows
@@ -80,6 +83,74 @@ def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, b
         cd.check()
         return _median(t_pre[1:]), _median(t_dec[1:])
 
+    def green_launches(q):
+        """Two green contexts that split the SMs (q for decode, the rest for prefill), one stream in each, the two
+        single-op launches released together.  Returns (prefill_us, decode_us, sms_decode, sms_prefill), or a string
+        saying why the driver would not make the contexts."""
+        try:
+            from cuda.bindings import driver as cu
+        except Exception as e:                      # pragma: no cover
+            return f"cuda-python not importable: {e}"
+        made = []
+        try:
+            err, cdev = cu.cuDeviceGet(dev.index or 0)
+            if err != cu.CUresult.CUDA_SUCCESS:
+                return f"cuDeviceGet: {err}"
+            err, res = cu.cuDeviceGetDevResource(cdev, cu.CUdevResourceType.CU_DEV_RESOURCE_TYPE_SM)
+            if err != cu.CUresult.CUDA_SUCCESS:
+                return f"cuDeviceGetDevResource: {err}"
+            err, groups, n_groups, rest = cu.cuDevSmResourceSplitByCount(1, res, 0, q)
+            if err != cu.CUresult.CUDA_SUCCESS or n_groups < 1:
+                return f"cuDevSmResourceSplitByCount: {err}"
+            streams, counts = [], []
+            for r in (groups[0], rest):
+                err, desc = cu.cuDevResourceGenerateDesc([r], 1)
+                if err != cu.CUresult.CUDA_SUCCESS:
+                    return f"cuDevResourceGenerateDesc: {err}"
+                err, g = cu.cuGreenCtxCreate(desc, cdev, cu.CUgreenCtxCreate_flags.CU_GREEN_CTX_DEFAULT_STREAM)
+                if err != cu.CUresult.CUDA_SUCCESS:
+                    return f"cuGreenCtxCreate: {err}"
+                made.append(g)
+                err, st = cu.cuGreenCtxStreamCreate(g, cu.CUstream_flags.CU_STREAM_NON_BLOCKING, 0)
+                if err != cu.CUresult.CUDA_SUCCESS:
+                    return f"cuGreenCtxStreamCreate: {err}"
+                streams.append(st)
+                counts.append(int(r.sm.smCount))
+            s_dec, s_pre = (torch.cuda.ExternalStream(int(st), device=dev) for st in streams)
+            n_dec, n_pre = counts[0] // 2 * 2, counts[1] // 2 * 2
+            cp = moe.Context(E, k, H, I, prefill_tokens, 1, n_ctas=n_pre, device=dev)
+            cd = moe.Context(E, k, H, I, decode_tokens, 1, n_ctas=n_dec, device=dev)
+            bp, bd = bind(cp, ops[0]), bind(cd, ops[1])
+            t_pre, t_dec = [], []
+            for _ in range(reps + 1):
+                cp.plan(0, bp)
+                cd.plan(0, bd)
+                torch.cuda.synchronize()
+                start = torch.cuda.Event(enable_timing=True)
+                ep = torch.cuda.Event(enable_timing=True)
+                ed = torch.cuda.Event(enable_timing=True)
+                start.record()
+                s_pre.wait_event(start)
+                s_dec.wait_event(start)
+                cp.run([0], fuse_combine=True, stream=s_pre)
+                ep.record(s_pre)
+                cd.run([0], fuse_combine=True, stream=s_dec)
+                ed.record(s_dec)
+                torch.cuda.synchronize()
+                t_pre.append(1e3 * start.elapsed_time(ep))
+                t_dec.append(1e3 * start.elapsed_time(ed))
+            cp.check()
+            cd.check()
+            for st in streams:
+                cu.cuStreamDestroy(st)
+            return _median(t_pre[1:]), _median(t_dec[1:]), counts[0], counts[1]
+        except Exception as e:
+            return f"{type(e).__name__}: {e}"
+        finally:
+            torch.cuda.synchronize()
+            for g in made:
+                cu.cuGreenCtxDestroy(g)
+
     def alone(op, tokens):
         c = moe.Context(E, k, H, I, tokens, 1, device=dev)
         b = bind(c, op)
@@ -127,6 +198,12 @@ def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, b
     for q in budgets:
         tp, td = two_launches(sms - q, q)
         rows.append(dict(arm="partition", q=q, prefill_us=tp, decode_us=td))
+    for q in budgets:
+        got = green_launches(q)
+        if isinstance(got, str):
+            rows.append(dict(arm="green", q=q, prefill_us=float("nan"), decode_us=float("nan"), unavailable=got))
+            break
+        rows.append(dict(arm="green", q=q, prefill_us=got[0], decode_us=got[1], sms_decode=got[2], sms_prefill=got[3]))
     for q in budgets:
         ta, td = apk(q)
         rows.append(dict(arm="apk", q=q, prefill_us=ta, decode_us=td))
@@ -207,8 +284,9 @@ def main():
         return
     rows = study()
     for r in rows:
-        print("%-13s q=%-4s prefill done %9.1f us   decode done %9.1f us" %
-              (r["arm"], "-" if r["q"] is None else r["q"], r["prefill_us"], r["decode_us"]))
+        print("%-13s q=%-4s prefill done %9.1f us   decode done %9.1f us  %s" %
+              (r["arm"], "-" if r["q"] is None else r["q"], r["prefill_us"], r["decode_us"],
+               r.get("unavailable", "") or ("SMs %d + %d" % (r["sms_decode"], r["sms_prefill"]) if "sms_decode" in r else "")))
     print(json.dumps(rows))
 
 
