@@ -23,6 +23,7 @@ launch the decode operation's completion comes from the kernel's tile log.
 launches of the same tile code, on a prefill-sized op and on decode-sized ops over 8..256 active experts.
 
     python -m paper_2607_18002_b200.sharing_study --overhead
+    python -m paper_2607_18002_b200.sharing_study --few-experts     # 8 192 prefill + 128 decode tokens on 8 experts
 """
 from __future__ import annotations
 
@@ -36,7 +37,10 @@ def _median(v):
 
 
 def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, budgets=(16, 32, 64, 96, 112, 128),
-          reps=5, seed=4, device="cuda:0"):
+          reps=5, seed=4, device="cuda:0", decode_active=None):
+    """decode_active: None routes the decode tokens by the same Zipf law as the prefill tokens (they then touch
+    most experts); a number confines them to a seeded pool of that many experts -- the regime of the paper's
+    experiment, where a decode batch meets few active experts on each GPU."""
     import torch
 
     import paper_2607_18002_b200 as moe
@@ -46,6 +50,9 @@ def study(E=256, k=8, H=3072, I=1536, prefill_tokens=16384, decode_tokens=256, b
                       "zipf", 1.0, 0.02, -1.0, seed)
     W = synth.make_weights(spec)
     ops = synth.make_ops(spec)
+    if decode_active is not None:
+        ids, w = synth.route_active_pool(np.random.default_rng([seed, 8]), decode_tokens, k, E, decode_active)
+        ops[1] = synth.Op(ops[1].cls, ops[1].x, ids, w, ops[1].x_scale)
     dev = torch.device(device)
     w1, w2 = W.w_gate_up.to(dev), W.w_down.to(dev)
     sms = torch.cuda.get_device_properties(dev).multi_processor_count
@@ -282,7 +289,10 @@ def main():
                    100.0 * (r["persistent_us"] / r["plain_us"] - 1.0), r["persistent_us"] - r["plain_us"]))
         print(json.dumps(rows))
         return
-    rows = study()
+    if "--few-experts" in sys.argv:      # the paper's setting: 8 192 prefill tokens next to 128 decode tokens on 8 experts
+        rows = study(prefill_tokens=8192, decode_tokens=128, decode_active=8, budgets=(16, 32, 64, 96, 128), reps=7)
+    else:
+        rows = study()
     for r in rows:
         print("%-13s q=%-4s prefill done %9.1f us   decode done %9.1f us  %s" %
               (r["arm"], "-" if r["q"] is None else r["q"], r["prefill_us"], r["decode_us"],
